@@ -1,0 +1,135 @@
+/*
+ * cowa.h -- C ABI of the CoWindow Attention (CoWA) library for NVIDIA B200 (sm_100a).
+ *
+ * The operator: causal grouped-query attention in which KV head h sees, for the
+ * query at bottom-right-aligned causal distance delta = i_q + (N_k - N_q) - i_k
+ * (Eq. fwa_distance), the union (Eq. fwa_support) of
+ *   near  { 0 <= delta < near }
+ *   sink  { i_k < sink, delta >= 0 }
+ *   long  { near + gap <= delta < near + gap + len }
+ * with one 4-tuple (sink, near, gap, len) per KV head (Sec. 2.1, after Eq. fwa_support).
+ * QO head h uses KV head floor(h * Hkv / Hq) and its tuple (GQA, Sec. 2.1).
+ *
+ * General conventions
+ *   - Every tensor pointer is a DEVICE pointer unless a comment says "host".
+ *   - q, k, v, o, d_o, dq, dk, dv are bf16; lse and workspaces are fp32/bytes.
+ *   - Default layout is contiguous head-major [B, H, T, D] with D innermost
+ *     (Algorithm 1/2 REQUIRE lines, plus a batch axis).  Base pointers must be
+ *     16-byte aligned.
+ *   - lse is the natural-log logsumexp of softmax_scale * q.k over the visible keys
+ *     (Algorithm 1 line 17), fp32 [B, Hq, T].
+ *   - The caller owns every buffer, workspaces included.  The library allocates no
+ *     device memory and keeps no state between calls except cached kernel
+ *     attributes.  All work is enqueued on `stream`; no call synchronises.
+ *   - Return value: COWA_OK (0) or a negative cowa_status_t.  Arguments are validated
+ *     before anything is launched.  There is no CPU fallback.
+ *   - Preconditions not checked on the device: near >= 1 for every head (so each
+ *     query sees at least its own position), lens[b] in [1, Tmax].
+ */
+#ifndef COWA_H_
+#define COWA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  COWA_OK = 0,
+  COWA_ERR_INVALID_ARG = -1,        /* null pointer, non-positive size, Hq % Hkv != 0, bad window */
+  COWA_ERR_UNSUPPORTED = -2,        /* D not in {64,128}; strides other than contiguous */
+  COWA_ERR_MISALIGNED = -3,         /* a base pointer is not 16-byte aligned */
+  COWA_ERR_WORKSPACE_TOO_SMALL = -4,
+  COWA_ERR_CUDA = -5,               /* a CUDA call failed; see cowa_last_cuda_error() */
+  COWA_ERR_DEVICE_TIMEOUT = -6      /* reported by cowa_check_device_status(): a bounded device wait ran out */
+} cowa_status_t;
+
+/* One KV head's windows: the paper's 4-tuple (sink width, near width, gap after the
+ * near window, long-range width), Sec. 2.1.  len == 0 means no long-range window. */
+typedef struct {
+  int32_t sink, near, gap, len;
+} cowa_window_t;
+
+typedef struct {
+  int32_t sink;        /* w_sink of the default rule (Eq. fwa_long_range_span) */
+  int32_t local;       /* w_near of the default rule; must be >= 1 */
+  int32_t block_q;     /* tile sizes used by cowa_schedule_dump (the kernels tile 128x128) */
+  int32_t block_k;
+  int32_t hkv_global;  /* global number of KV heads (Eq. fwa_global_head); 0 => Hkv */
+  int32_t hkv_offset;  /* global index of this call's KV head 0; 0 on one GPU */
+  const cowa_window_t* windows; /* HOST pointer to Hkv explicit tuples, or NULL for the default rule.
+                                   Read during the call; not retained.  Ignored by cowa_decode. */
+  int32_t full_attn;   /* 1 => every head sees the whole causal prefix (dense FullAttn path) */
+  float softmax_scale; /* scores are softmax_scale * q.k (the paper pre-scales Q by 1/sqrt(d_h)) */
+} cowa_params_t;
+
+/* Training / prefill forward, Algorithm 1.  N_q = N_k = T.
+ *   q [B,Hq,T,D], k,v [B,Hkv,T,D] in; o [B,Hq,T,D] bf16 and lse [B,Hq,T] fp32 out.
+ * D in {64,128}; Hq a multiple of Hkv.  No workspace. */
+int cowa_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
+             int B, int T, int Hq, int Hkv, int D, const cowa_params_t* p, void* stream);
+
+/* Training backward, Algorithm 2: exact gradient of cowa_fwd.
+ *   in: q,k,v,o,lse as produced by cowa_fwd, d_o [B,Hq,T,D];
+ *   out: dq [B,Hq,T,D], dk,dv [B,Hkv,T,D] bf16 (fully overwritten).
+ * dk,dv are summed over the QO heads of each group inside one thread block (no atomics);
+ * `workspace` (device, >= cowa_bwd_workspace_bytes, 16-byte aligned) holds the fp32
+ * row vector rowsum(o*d_o) (Algorithm 2 line 13) and needs no initialisation. */
+int cowa_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse,
+             const void* d_o, void* dq, void* dk, void* dv,
+             int B, int T, int Hq, int Hkv, int D, const cowa_params_t* p,
+             void* workspace, size_t workspace_bytes, void* stream);
+
+/* Single-token decode over a KV cache (Sec. 2.3 "Decoding"): the forward with N_q = 1.
+ *   q [B,Hq,D]; kcache,vcache [B,Hkv,Tmax,D]; lens int32 [B] on the DEVICE, lens[b] = N_k
+ *   = cached tokens + 1, the current token's K/V already stored at index lens[b]-1.
+ *   Breakpoints are recomputed from lens[b] for every sequence (default rule only).
+ *   out: o [B,Hq,D] bf16; lse [B,Hq] fp32 (may be NULL).
+ * Only the visible rows of each head are read.  Split-KV partial states go to `workspace`
+ * (device, >= cowa_decode_workspace_bytes, 16-byte aligned, no initialisation needed) and
+ * are merged by a second kernel on the same stream. */
+int cowa_decode(const void* q, const void* kcache, const void* vcache, const int32_t* lens,
+                void* o, float* lse, int B, int Tmax, int Hq, int Hkv, int D,
+                const cowa_params_t* p, void* workspace, size_t workspace_bytes, void* stream);
+
+size_t cowa_bwd_workspace_bytes(int B, int T, int Hq, int Hkv, int D, const cowa_params_t* p);
+size_t cowa_decode_workspace_bytes(int B, int Tmax, int Hq, int Hkv, int D, const cowa_params_t* p);
+
+/* Host-only.  Default 4-tuples (sink, local, b_h, b_{h+1}-b_h), b_h = floor(h*L/Hkv_global),
+ * L = max(Nk - sink - local, 0), for global heads hkv_offset .. hkv_offset+Hkv_local-1
+ * (Eq. fwa_long_range_span, Eq. fwa_global_head).  out: HOST array of Hkv_local tuples. */
+int cowa_default_windows(int Nk, int Hkv_global, int hkv_offset, int Hkv_local,
+                         int sink, int local, cowa_window_t* out);
+
+/* Host-only.  Writes the analytic tile schedule (Sec. 2.3: block sets J_h(i), I_h(j)) that the
+ * kernels' scheduler computes, as an int32 stream into the HOST buffer `out`:
+ *   COWA_SCHED_FWD    for each head h, QO tile i:  h, i, n, then n pairs (j, full) with j descending
+ *   COWA_SCHED_BWD    for each head h, KV tile j:  h, j, n, then n pairs (i, full) with i ascending
+ *   COWA_SCHED_DECODE (Nq must be 1) for each head h: h, r, then r pairs (start, end) of visible key
+ *                     ranges [start,end) ascending, then m, then m visited block_k-block indices
+ * full = 1 when every pair of the nominal block_q x block_k tile is legal, else 0 (boundary tile).
+ * *out_len receives the number of int32 needed; COWA_ERR_WORKSPACE_TOO_SMALL if out_cap is less
+ * (nothing beyond out_cap is written). */
+enum { COWA_SCHED_FWD = 0, COWA_SCHED_BWD = 1, COWA_SCHED_DECODE = 2 };
+int cowa_schedule_dump(int which, int Nq, int Nk, int Hkv, const cowa_params_t* p,
+                       int32_t* out, size_t out_cap, size_t* out_len);
+
+/* Visited-tile counts of the 128x128 kernel tiling summed over the Hkv heads (host-only):
+ * out[0] = visited, out[1] = full, out[2] = causal tiles.  Used for FLOP accounting. */
+int cowa_tile_counts(int Nq, int Nk, int Hkv, const cowa_params_t* p, int64_t out[3]);
+
+/* The kernels bound every device-side wait; a wait that runs out sets a flag in a device word
+ * instead of hanging.  This call synchronises `stream`, reads and clears the flag, and returns
+ * COWA_OK or COWA_ERR_DEVICE_TIMEOUT (COWA_ERR_CUDA if the stream itself reports an error). */
+int cowa_check_device_status(void* stream);
+
+const char* cowa_status_string(int status);
+/* cudaError_t value of the most recent failing CUDA call made by this library on this thread. */
+int cowa_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COWA_H_ */

@@ -1,0 +1,190 @@
+"""ctypes binding of include/cowa.h.  Function names equal the C entry points.
+
+The shared library must have been built (python -m paper_2609_32704_b200.build or
+__graft_entry__.build()); there is no fallback when it is missing.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+lib_path = os.path.join(_HERE, "libcowa.so")
+
+SCHED_FWD, SCHED_BWD, SCHED_DECODE = 0, 1, 2
+
+
+class CowaError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        msg = lib().cowa_status_string(status).decode()
+        extra = f" (cudaError {lib().cowa_last_cuda_error()})" if status == -5 else ""
+        super().__init__(f"{where}: {msg}{extra} [{status}]")
+
+
+class Window(C.Structure):
+    _fields_ = [("sink", C.c_int32), ("near", C.c_int32), ("gap", C.c_int32), ("len", C.c_int32)]
+
+
+class Params(C.Structure):
+    _fields_ = [
+        ("sink", C.c_int32), ("local", C.c_int32), ("block_q", C.c_int32), ("block_k", C.c_int32),
+        ("hkv_global", C.c_int32), ("hkv_offset", C.c_int32), ("windows", C.POINTER(Window)),
+        ("full_attn", C.c_int32), ("softmax_scale", C.c_float),
+    ]
+
+
+_lib = None
+
+
+def lib():
+    """The loaded C library (raises if it has not been built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(lib_path):
+            raise ImportError(f"{lib_path} not found: build it with `python -m paper_2609_32704_b200.build`")
+        L = C.CDLL(lib_path)
+        vp, i32, sz = C.c_void_p, C.c_int, C.c_size_t
+        pp = C.POINTER(Params)
+        L.cowa_fwd.argtypes = [vp] * 5 + [i32] * 5 + [pp, vp]
+        L.cowa_fwd.restype = i32
+        L.cowa_bwd.argtypes = [vp] * 9 + [i32] * 5 + [pp, vp, sz, vp]
+        L.cowa_bwd.restype = i32
+        L.cowa_decode.argtypes = [vp] * 6 + [i32] * 5 + [pp, vp, sz, vp]
+        L.cowa_decode.restype = i32
+        L.cowa_bwd_workspace_bytes.argtypes = [i32] * 5 + [pp]
+        L.cowa_bwd_workspace_bytes.restype = sz
+        L.cowa_decode_workspace_bytes.argtypes = [i32] * 5 + [pp]
+        L.cowa_decode_workspace_bytes.restype = sz
+        L.cowa_default_windows.argtypes = [i32] * 6 + [C.POINTER(Window)]
+        L.cowa_default_windows.restype = i32
+        L.cowa_schedule_dump.argtypes = [i32, i32, i32, i32, pp, C.POINTER(C.c_int32), sz, C.POINTER(sz)]
+        L.cowa_schedule_dump.restype = i32
+        L.cowa_tile_counts.argtypes = [i32, i32, i32, pp, C.POINTER(C.c_int64)]
+        L.cowa_tile_counts.restype = i32
+        L.cowa_check_device_status.argtypes = [vp]
+        L.cowa_check_device_status.restype = i32
+        L.cowa_status_string.argtypes = [i32]
+        L.cowa_status_string.restype = C.c_char_p
+        L.cowa_last_cuda_error.argtypes = []
+        L.cowa_last_cuda_error.restype = i32
+        _lib = L
+    return _lib
+
+
+def make_params(sink=0, local=1, block=128, softmax_scale=1.0, windows=None, full_attn=False,
+                hkv_global=0, hkv_offset=0, block_q=None, block_k=None):
+    """Fills a cowa_params_t.  `windows`: optional list of (sink, near, gap, len) per KV head."""
+    p = Params()
+    p.sink, p.local = int(sink), int(local)
+    p.block_q = int(block_q if block_q is not None else block)
+    p.block_k = int(block_k if block_k is not None else block)
+    p.hkv_global, p.hkv_offset = int(hkv_global), int(hkv_offset)
+    p.full_attn = 1 if full_attn else 0
+    p.softmax_scale = float(softmax_scale)
+    if windows is not None:
+        arr = (Window * len(windows))(*[Window(*map(int, w)) for w in windows])
+        p.windows = C.cast(arr, C.POINTER(Window))
+        p._keepalive = arr
+    return p
+
+
+def _check(status, where):
+    if status != 0:
+        raise CowaError(status, where)
+
+
+def _stream():
+    import torch
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _ptr(t):
+    return C.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _need(t, dtype, name):
+    import torch
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous() and t.dtype == dtype):
+        raise TypeError(f"{name}: expected a contiguous CUDA tensor of {dtype}")
+
+
+def cowa_fwd(q, k, v, o, lse, params):
+    """q [B,Hq,T,D], k/v [B,Hkv,T,D] bf16 -> o (bf16), lse (fp32 [B,Hq,T]); all preallocated."""
+    import torch
+    for t, n in ((q, "q"), (k, "k"), (v, "v"), (o, "o")):
+        _need(t, torch.bfloat16, n)
+    _need(lse, torch.float32, "lse")
+    B, Hq, T, D = q.shape
+    Hkv = k.shape[1]
+    _check(lib().cowa_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), B, T, Hq, Hkv, D,
+                          C.byref(params), _stream()), "cowa_fwd")
+
+
+def cowa_bwd_workspace_bytes(B, T, Hq, Hkv, D, params):
+    return int(lib().cowa_bwd_workspace_bytes(B, T, Hq, Hkv, D, C.byref(params)))
+
+
+def cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, params, workspace):
+    """Gradients dq, dk, dv (bf16, preallocated) of cowa_fwd; workspace: uint8 CUDA tensor."""
+    import torch
+    for t, n in ((q, "q"), (k, "k"), (v, "v"), (o, "o"), (d_o, "d_o"), (dq, "dq"), (dk, "dk"), (dv, "dv")):
+        _need(t, torch.bfloat16, n)
+    _need(lse, torch.float32, "lse")
+    B, Hq, T, D = q.shape
+    Hkv = k.shape[1]
+    _check(lib().cowa_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(d_o), _ptr(dq), _ptr(dk),
+                          _ptr(dv), B, T, Hq, Hkv, D, C.byref(params), _ptr(workspace),
+                          workspace.numel() * workspace.element_size(), _stream()), "cowa_bwd")
+
+
+def cowa_decode_workspace_bytes(B, Tmax, Hq, Hkv, D, params):
+    return int(lib().cowa_decode_workspace_bytes(B, Tmax, Hq, Hkv, D, C.byref(params)))
+
+
+def cowa_decode(q, kcache, vcache, lens, o, lse, params, workspace):
+    """q [B,Hq,D], caches [B,Hkv,Tmax,D] bf16, lens int32 [B] (device) -> o [B,Hq,D], lse [B,Hq] or None."""
+    import torch
+    for t, n in ((q, "q"), (kcache, "kcache"), (vcache, "vcache"), (o, "o")):
+        _need(t, torch.bfloat16, n)
+    _need(lens, torch.int32, "lens")
+    if lse is not None:
+        _need(lse, torch.float32, "lse")
+    B, Hq, D = q.shape
+    Hkv, Tmax = kcache.shape[1], kcache.shape[2]
+    _check(lib().cowa_decode(_ptr(q), _ptr(kcache), _ptr(vcache), _ptr(lens), _ptr(o), _ptr(lse), B, Tmax,
+                             Hq, Hkv, D, C.byref(params), _ptr(workspace),
+                             workspace.numel() * workspace.element_size(), _stream()), "cowa_decode")
+
+
+def cowa_default_windows(Nk, Hkv_global, hkv_offset, Hkv_local, sink, local):
+    out = (Window * Hkv_local)()
+    _check(lib().cowa_default_windows(Nk, Hkv_global, hkv_offset, Hkv_local, sink, local, out),
+           "cowa_default_windows")
+    return [(w.sink, w.near, w.gap, w.len) for w in out]
+
+
+def cowa_schedule_dump(which, Nq, Nk, Hkv, params):
+    """Returns the int32 stream described in cowa.h as a list."""
+    n = C.c_size_t(0)
+    st = lib().cowa_schedule_dump(which, Nq, Nk, Hkv, C.byref(params), None, 0, C.byref(n))
+    if st not in (0, -4):
+        _check(st, "cowa_schedule_dump")
+    buf = (C.c_int32 * max(n.value, 1))()
+    _check(lib().cowa_schedule_dump(which, Nq, Nk, Hkv, C.byref(params), buf, n.value, C.byref(n)),
+           "cowa_schedule_dump")
+    return list(buf[:n.value])
+
+
+def cowa_tile_counts(Nq, Nk, Hkv, params):
+    out = (C.c_int64 * 3)()
+    _check(lib().cowa_tile_counts(Nq, Nk, Hkv, C.byref(params), out), "cowa_tile_counts")
+    return dict(visited=out[0], full=out[1], causal=out[2])
+
+
+def cowa_check_device_status():
+    _check(lib().cowa_check_device_status(_stream()), "cowa_check_device_status")
+
+
+def cowa_status_string(status):
+    return lib().cowa_status_string(status).decode()

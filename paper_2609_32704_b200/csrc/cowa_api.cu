@@ -1,0 +1,190 @@
+// Host-side pieces of the C ABI that launch nothing: window resolution, the schedule dump,
+// tile counts, status reporting.
+#include <string.h>
+
+#include "cowa_common.h"
+
+namespace {
+thread_local int g_last_cuda_error = 0;
+__device__ unsigned int g_cowa_status_word = 0;
+}  // namespace
+
+namespace cowa {
+
+int record_cuda_error(cudaError_t e) {
+  g_last_cuda_error = (int)e;
+  return COWA_ERR_CUDA;
+}
+
+unsigned int* device_status_word() {
+  // One address per device; looked up once per device with that device current.
+  static unsigned int* cache[64] = {nullptr};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (!cache[dev]) {
+    void* ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&ptr, g_cowa_status_word);
+    if (e != cudaSuccess) { record_cuda_error(e); return nullptr; }
+    cache[dev] = static_cast<unsigned int*>(ptr);
+  }
+  return cache[dev];
+}
+
+int resolve_windows(int Nk, int Hkv, const cowa_params_t* p, CowaHeadWindows* out) {
+  if (!p || Hkv <= 0 || Nk <= 0) return COWA_ERR_INVALID_ARG;
+  if (Hkv > COWA_MAX_HKV) return COWA_ERR_UNSUPPORTED;
+  const int hg = p->hkv_global > 0 ? p->hkv_global : Hkv;
+  if (p->hkv_offset < 0 || p->hkv_offset + Hkv > hg) return COWA_ERR_INVALID_ARG;
+  for (int h = 0; h < Hkv; ++h) {
+    CowaWin w;
+    if (p->full_attn) {
+      w.s = 0; w.n = Nk; w.g = 0; w.l = 0;  // near window spans the whole prefix
+    } else if (p->windows) {
+      const cowa_window_t& t = p->windows[h];
+      if (t.sink < 0 || t.near < 1 || t.gap < 0 || t.len < 0) return COWA_ERR_INVALID_ARG;
+      w.s = t.sink; w.n = t.near; w.g = t.gap; w.l = t.len;
+    } else {
+      if (p->sink < 0 || p->local < 1) return COWA_ERR_INVALID_ARG;
+      w = cowa_default_window(Nk, hg, p->hkv_offset + h, p->sink, p->local);
+    }
+    out->w[h] = w;
+  }
+  return COWA_OK;
+}
+
+}  // namespace cowa
+
+extern "C" {
+
+int cowa_default_windows(int Nk, int Hkv_global, int hkv_offset, int Hkv_local, int sink, int local,
+                         cowa_window_t* out) {
+  if (!out || Nk <= 0 || Hkv_global <= 0 || Hkv_local <= 0 || hkv_offset < 0 ||
+      hkv_offset + Hkv_local > Hkv_global || sink < 0 || local < 1)
+    return COWA_ERR_INVALID_ARG;
+  for (int h = 0; h < Hkv_local; ++h) {
+    CowaWin w = cowa_default_window(Nk, Hkv_global, hkv_offset + h, sink, local);
+    out[h].sink = w.s; out[h].near = w.n; out[h].gap = w.g; out[h].len = w.l;
+  }
+  return COWA_OK;
+}
+
+int cowa_schedule_dump(int which, int Nq, int Nk, int Hkv, const cowa_params_t* p, int32_t* out,
+                       size_t out_cap, size_t* out_len) {
+  if (!p || !out_len || Nq <= 0 || Nk <= 0 || Nq > Nk || Hkv <= 0) return COWA_ERR_INVALID_ARG;
+  if (p->block_q <= 0 || p->block_k <= 0) return COWA_ERR_INVALID_ARG;
+  if (which == COWA_SCHED_DECODE && Nq != 1) return COWA_ERR_INVALID_ARG;
+  if (Hkv > COWA_MAX_HKV) return COWA_ERR_UNSUPPORTED;
+  CowaHeadWindows hw;
+  int st = cowa::resolve_windows(Nk, Hkv, p, &hw);
+  if (st != COWA_OK) return st;
+  const int Bq = p->block_q, Bk = p->block_k, off = Nk - Nq;
+  const int Tq = (Nq + Bq - 1) / Bq, Tk = (Nk + Bk - 1) / Bk;
+  size_t n = 0;
+  auto put = [&](int32_t x) {
+    if (out && n < out_cap) out[n] = x;
+    ++n;
+  };
+  for (int h = 0; h < Hkv; ++h) {
+    const CowaWin& w = hw.w[h];
+    if (which == COWA_SCHED_FWD) {
+      for (int i = 0; i < Tq; ++i) {
+        const int q0 = i * Bq, q1 = cowa_imin(q0 + Bq, Nq) - 1;
+        CowaRange r[3];
+        cowa_fwd_ranges(w, q0, q1, off, Nk, Bk, r);
+        const int tot = cowa_range_len(r[0]) + cowa_range_len(r[1]) + cowa_range_len(r[2]);
+        put(h); put(i); put(tot);
+        for (int t = 0; t < tot; ++t) {
+          const int j = cowa_fwd_tile_at(r, t);
+          put(j);
+          put(cowa_tile_full(w, q0, Bq, j * Bk, Bk, off, Nq, Nk) ? 1 : 0);
+        }
+      }
+    } else if (which == COWA_SCHED_BWD) {
+      for (int j = 0; j < Tk; ++j) {
+        const int k0 = j * Bk, k1 = cowa_imin(k0 + Bk, Nk) - 1;
+        CowaRange r[2];
+        cowa_bwd_ranges(w, k0, k1, off, Nq, Bq, r);
+        const int tot = cowa_range_len(r[0]) + cowa_range_len(r[1]);
+        put(h); put(j); put(tot);
+        for (int t = 0; t < tot; ++t) {
+          const int i = cowa_bwd_tile_at(r, t);
+          put(i);
+          put(cowa_tile_full(w, i * Bq, Bq, k0, Bk, off, Nq, Nk) ? 1 : 0);
+        }
+      }
+    } else if (which == COWA_SCHED_DECODE) {
+      CowaRange r[3];
+      const int nr = cowa_decode_ranges(w, Nk, r);
+      put(h); put(nr);
+      for (int t = 0; t < nr; ++t) { put(r[t].lo); put(r[t].hi + 1); }
+      // visited blocks: the blocks touched by the ranges, each once
+      size_t cnt_at = n;
+      put(0);
+      int32_t cnt = 0;
+      int last = -1;
+      for (int t = 0; t < nr; ++t) {
+        for (int b = cowa_imax(r[t].lo / Bk, last + 1); b <= r[t].hi / Bk; ++b) { put(b); ++cnt; last = b; }
+      }
+      if (out && cnt_at < out_cap) out[cnt_at] = cnt;
+    } else {
+      return COWA_ERR_INVALID_ARG;
+    }
+  }
+  *out_len = n;
+  return (out && n <= out_cap) ? COWA_OK : COWA_ERR_WORKSPACE_TOO_SMALL;
+}
+
+int cowa_tile_counts(int Nq, int Nk, int Hkv, const cowa_params_t* p, int64_t out[3]) {
+  if (!p || !out || Nq <= 0 || Nk <= 0 || Nq > Nk || Hkv <= 0) return COWA_ERR_INVALID_ARG;
+  CowaHeadWindows hw;
+  int st = cowa::resolve_windows(Nk, Hkv, p, &hw);
+  if (st != COWA_OK) return st;
+  const int B = 128, off = Nk - Nq, Tq = (Nq + B - 1) / B;
+  int64_t visited = 0, full = 0, causal = 0;
+  for (int h = 0; h < Hkv; ++h) {
+    for (int i = 0; i < Tq; ++i) {
+      const int q0 = i * B, q1 = cowa_imin(q0 + B, Nq) - 1;
+      CowaRange r[3];
+      cowa_fwd_ranges(hw.w[h], q0, q1, off, Nk, B, r);
+      const int tot = cowa_range_len(r[0]) + cowa_range_len(r[1]) + cowa_range_len(r[2]);
+      visited += tot;
+      for (int t = 0; t < tot; ++t)
+        full += cowa_tile_full(hw.w[h], q0, B, cowa_fwd_tile_at(r, t) * B, B, off, Nq, Nk) ? 1 : 0;
+      causal += cowa_imin(q1 + off, Nk - 1) / B + 1;
+    }
+  }
+  out[0] = visited; out[1] = full; out[2] = causal;
+  return COWA_OK;
+}
+
+int cowa_check_device_status(void* stream) {
+  unsigned int* word = cowa::device_status_word();
+  if (!word) return COWA_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  unsigned int host = 0;
+  COWA_CUDA_TRY(cudaMemcpyAsync(&host, word, sizeof(host), cudaMemcpyDeviceToHost, s));
+  COWA_CUDA_TRY(cudaStreamSynchronize(s));
+  if (host != 0) {
+    COWA_CUDA_TRY(cudaMemsetAsync(word, 0, sizeof(host), s));
+    COWA_CUDA_TRY(cudaStreamSynchronize(s));
+    return COWA_ERR_DEVICE_TIMEOUT;
+  }
+  return COWA_OK;
+}
+
+const char* cowa_status_string(int status) {
+  switch (status) {
+    case COWA_OK: return "ok";
+    case COWA_ERR_INVALID_ARG: return "invalid argument";
+    case COWA_ERR_UNSUPPORTED: return "unsupported configuration";
+    case COWA_ERR_MISALIGNED: return "pointer not 16-byte aligned";
+    case COWA_ERR_WORKSPACE_TOO_SMALL: return "workspace or output buffer too small";
+    case COWA_ERR_CUDA: return "CUDA call failed";
+    case COWA_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+    default: return "unknown status";
+  }
+}
+
+int cowa_last_cuda_error(void) { return g_last_cuda_error; }
+
+}  // extern "C"

@@ -1,0 +1,373 @@
+// Split-KV single-token decode for CoWindow Attention (Sec. 2.3 "Decoding"): the forward
+// with N_q = 1, delta = N_k - 1 - i_k, windows recomputed from the current key length of each
+// sequence; the visible rows of a head are divided over split programs whose partial
+// online-softmax states are merged afterwards.
+//
+// HBM-bound: every visible K and V row is read exactly once, with 128-bit loads, straight
+// into registers.  Per (sequence, KV head, split) one 128-thread block:
+//   1. scores:  each warp takes 16 visible rows at a time; K rows are loaded as the A
+//      fragment of mma.sync m16n8k16 (bf16, fp32 accumulate), the group's query vectors are
+//      the B fragment.  The contraction index is permuted identically on both operands so
+//      that every thread's loads are 16-byte vectors.  Scores (log2 units) go to shared memory.
+//   2. block-wide max / exp2 / sum per QO head (no running rescale: the split's scores are
+//      all in shared memory before any V row is touched).
+//   3. values:  thread = (8-wide slice of D, row subgroup); fp32 FMAs over the split's V rows
+//      with the probabilities broadcast from shared memory; row subgroups reduced in shared
+//      memory; un-normalised partial (o, m, l) written to the workspace.
+// A second kernel merges the splits (log-sum-exp combine with warp shuffles).
+#include <cuda_bf16.h>
+
+#include "cowa_common.h"
+
+namespace {
+
+constexpr int kThreads = 128;
+constexpr int kChunkCap = 1024;  // max visible rows per split (scores of a split live in shared memory)
+
+struct DecodeArgs {
+  const __nv_bfloat16* q;
+  const __nv_bfloat16* kc;
+  const __nv_bfloat16* vc;
+  const int32_t* lens;
+  float* ws_o;  // [B, Hq, S, D]
+  float* ws_m;  // [B, Hq, S]
+  float* ws_l;  // [B, Hq, S]
+  int B, Tmax, Hq, Hkv, S;
+  int sink, near, hkv_global, hkv_offset, full_attn;
+  float scale_log2;
+};
+
+// Position of the v-th visible row (v in the concatenation of the head's ranges).
+struct VisMap {
+  int lo0, n0, lo1, n1, lo2;
+  __device__ __forceinline__ int token(int v) const {
+    return v < n0 ? lo0 + v : (v < n0 + n1 ? lo1 + (v - n0) : lo2 + (v - n0 - n1));
+  }
+};
+
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                               uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};\n"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint4 ldg128(const void* p) {
+  uint4 r;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+               : "l"(p));
+  return r;
+}
+
+__device__ __forceinline__ float bf16lo(uint32_t x) { return __uint_as_float(x << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t x) { return __uint_as_float(x & 0xffff0000u); }
+
+template <int D, int G>
+__global__ void __launch_bounds__(kThreads) cowa_decode_split_kernel(const DecodeArgs a) {
+  static_assert(D == 64 || D == 128, "head dim");
+  static_assert(G >= 1 && G <= 8, "group size per mma n-tile");
+  constexpr int DC = D / 8;           // 16-byte slices per row
+  constexpr int RP = kThreads / DC;   // rows handled in parallel in the value phase
+  constexpr int KC = D / 32;          // 32-wide d chunks (two k16 steps each)
+
+  __shared__ __align__(16) float sc[G * kChunkCap];  // scores, later the value-phase reduction buffer
+  __shared__ float m_s[G], l_s[G];
+
+  const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int Nk = a.lens[b];
+
+  // visible ranges of this head for the current key length
+  CowaWin w;
+  if (a.full_attn) { w.s = 0; w.n = Nk; w.g = 0; w.l = 0; }
+  else w = cowa_default_window(Nk, a.hkv_global, a.hkv_offset + hk, a.sink, a.near);
+  CowaRange rg[3];
+  const int nr = cowa_decode_ranges(w, Nk, rg);
+  VisMap vm;
+  vm.lo0 = rg[0].lo; vm.n0 = nr > 0 ? rg[0].hi - rg[0].lo + 1 : 0;
+  vm.lo1 = nr > 1 ? rg[1].lo : 0; vm.n1 = nr > 1 ? rg[1].hi - rg[1].lo + 1 : 0;
+  vm.lo2 = nr > 2 ? rg[2].lo : 0;
+  const int n2 = nr > 2 ? rg[2].hi - rg[2].lo + 1 : 0;
+  const int V = vm.n0 + vm.n1 + n2;
+
+  int chunk = (V + a.S - 1) / a.S;
+  chunk = (chunk + 15) & ~15;
+  const int c0 = split * chunk;
+  const int clen = min(chunk, V - c0);  // <= kChunkCap by the host's choice of S
+
+  const size_t head0 = (size_t)b * a.Hq + (size_t)hk * G;
+  if (clen <= 0) {  // empty split: neutral partial state
+    for (int i = tid; i < G * D; i += kThreads)
+      a.ws_o[((head0 + i / D) * a.S + split) * D + (i % D)] = 0.f;
+    if (tid < G) {
+      a.ws_m[(head0 + tid) * a.S + split] = -INFINITY;
+      a.ws_l[(head0 + tid) * a.S + split] = 0.f;
+    }
+    return;
+  }
+
+  const __nv_bfloat16* kbase = a.kc + ((size_t)b * a.Hkv + hk) * (size_t)a.Tmax * D;
+  const __nv_bfloat16* vbase = a.vc + ((size_t)b * a.Hkv + hk) * (size_t)a.Tmax * D;
+
+  // ---------------- phase 1: scores ----------------
+  {
+    const int g = lane >> 2, t = lane & 3;
+    // B fragments: query head g (zero beyond the group), permuted contraction index
+    uint32_t bq[KC][4];
+#pragma unroll
+    for (int cc = 0; cc < KC; ++cc) {
+      uint4 x = make_uint4(0, 0, 0, 0);
+      if (g < G) x = *reinterpret_cast<const uint4*>(a.q + (head0 + g) * D + cc * 32 + t * 8);
+      bq[cc][0] = x.x; bq[cc][1] = x.y; bq[cc][2] = x.z; bq[cc][3] = x.w;
+    }
+    const int nblk = (clen + 15) >> 4;
+    for (int blk = warp; blk < nblk; blk += kThreads / 32) {
+      const int rA = blk * 16 + g, rB = rA + 8;
+      const int tokA = vm.token(c0 + min(rA, clen - 1));
+      const int tokB = vm.token(c0 + min(rB, clen - 1));
+      const __nv_bfloat16* pa = kbase + (size_t)tokA * D + t * 8;
+      const __nv_bfloat16* pb = kbase + (size_t)tokB * D + t * 8;
+      uint4 ka[KC], kb[KC];
+#pragma unroll
+      for (int cc = 0; cc < KC; ++cc) { ka[cc] = ldg128(pa + cc * 32); kb[cc] = ldg128(pb + cc * 32); }
+      float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int cc = 0; cc < KC; ++cc) {
+        mma_bf16_16816(c, ka[cc].x, kb[cc].x, ka[cc].y, kb[cc].y, bq[cc][0], bq[cc][1]);
+        mma_bf16_16816(c, ka[cc].z, kb[cc].z, ka[cc].w, kb[cc].w, bq[cc][2], bq[cc][3]);
+      }
+      // c[0],c[1]: row rA, heads 2t, 2t+1;  c[2],c[3]: row rB
+      const int h0 = 2 * t, h1 = 2 * t + 1;
+      if (rA < clen) {
+        if (h0 < G) sc[h0 * kChunkCap + rA] = c[0] * a.scale_log2;
+        if (h1 < G) sc[h1 * kChunkCap + rA] = c[1] * a.scale_log2;
+      }
+      if (rB < clen) {
+        if (h0 < G) sc[h0 * kChunkCap + rB] = c[2] * a.scale_log2;
+        if (h1 < G) sc[h1 * kChunkCap + rB] = c[3] * a.scale_log2;
+      }
+    }
+  }
+  __syncthreads();
+
+  // ---------------- phase 2: max, exp2, sum per head ----------------
+  for (int h = warp; h < G; h += kThreads / 32) {
+    float* s = sc + h * kChunkCap;
+    float m = -INFINITY;
+    for (int r = lane; r < clen; r += 32) m = fmaxf(m, s[r]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    float l = 0.f;
+    for (int r = lane; r < clen; r += 32) {
+      float p = exp2f(s[r] - m);
+      s[r] = p;
+      l += p;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+    if (lane == 0) { m_s[h] = m; l_s[h] = l; }
+  }
+  __syncthreads();
+
+  // ---------------- phase 3: values ----------------
+  const int dch = tid % DC, rs = tid / DC;
+  float acc[G][8];
+#pragma unroll
+  for (int h = 0; h < G; ++h)
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[h][i] = 0.f;
+
+  constexpr int U = 4;
+  for (int r0 = rs; r0 < clen; r0 += RP * U) {
+    uint4 vv[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int r = min(r0 + u * RP, clen - 1);
+      vv[u] = ldg128(vbase + (size_t)vm.token(c0 + r) * D + dch * 8);
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int r = r0 + u * RP;
+      if (r < clen) {
+        float x[8] = {bf16lo(vv[u].x), bf16hi(vv[u].x), bf16lo(vv[u].y), bf16hi(vv[u].y),
+                      bf16lo(vv[u].z), bf16hi(vv[u].z), bf16lo(vv[u].w), bf16hi(vv[u].w)};
+#pragma unroll
+        for (int h = 0; h < G; ++h) {
+          const float p = sc[h * kChunkCap + r];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) acc[h][i] = fmaf(p, x[i], acc[h][i]);
+        }
+      }
+    }
+  }
+  __syncthreads();  // scores no longer needed: reuse as red[rs][h][d]  (RP * D == kChunkCap)
+  static_assert(RP * D <= kChunkCap, "reduction buffer fits the score buffer");
+#pragma unroll
+  for (int h = 0; h < G; ++h) {
+    float4* dst = reinterpret_cast<float4*>(sc + ((size_t)(rs * G + h) * D + dch * 8));
+    dst[0] = make_float4(acc[h][0], acc[h][1], acc[h][2], acc[h][3]);
+    dst[1] = make_float4(acc[h][4], acc[h][5], acc[h][6], acc[h][7]);
+  }
+  __syncthreads();
+  for (int i = tid; i < G * D; i += kThreads) {
+    float s = 0.f;
+#pragma unroll
+    for (int r = 0; r < RP; ++r) s += sc[r * G * D + i];
+    a.ws_o[((head0 + i / D) * a.S + split) * D + (i % D)] = s;
+  }
+  if (tid < G) {
+    a.ws_m[(head0 + tid) * a.S + split] = m_s[tid];
+    a.ws_l[(head0 + tid) * a.S + split] = l_s[tid];
+  }
+}
+
+// Merge of the split states: M = max m_s, L = sum l_s 2^(m_s - M), o = sum o_s 2^(m_s - M) / L,
+// lse = ln2 * (M + log2 L).  One block per (sequence, QO head), D threads.
+template <int D>
+__global__ void __launch_bounds__(D) cowa_decode_combine_kernel(const float* __restrict__ ws_o,
+                                                                const float* __restrict__ ws_m,
+                                                                const float* __restrict__ ws_l,
+                                                                __nv_bfloat16* __restrict__ o,
+                                                                float* __restrict__ lse, int S) {
+  const size_t bh = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31;
+  const float* m = ws_m + bh * S;
+  const float* l = ws_l + bh * S;
+  float mx = -INFINITY;
+  for (int s = lane; s < S; s += 32) mx = fmaxf(mx, m[s]);
+#pragma unroll
+  for (int o_ = 16; o_ > 0; o_ >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o_));
+  float L = 0.f;
+  for (int s = lane; s < S; s += 32) L += l[s] * exp2f(m[s] - mx);  // empty splits: l = 0, m = -inf -> 0
+#pragma unroll
+  for (int o_ = 16; o_ > 0; o_ >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o_);
+  float acc = 0.f;
+  const float* po = ws_o + bh * S * D + tid;
+  for (int s = 0; s < S; ++s) acc = fmaf(po[(size_t)s * D], exp2f(m[s] - mx), acc);
+  o[bh * D + tid] = __float2bfloat16_rn(acc / L);
+  if (lse && tid == 0) lse[bh] = 0.6931471805599453f * (mx + log2f(L));
+}
+
+// Upper bound of visible rows per head for any key length <= Tmax.
+int max_visible(int Tmax, int hg, const cowa_params_t* p) {
+  if (p->full_attn) return Tmax;
+  long long shared = (long long)p->sink + p->local;
+  if (shared >= Tmax) return Tmax;
+  long long band = ((long long)Tmax - shared + hg - 1) / hg;  // widest band, ceil(L / Hk)
+  long long v = shared + band;
+  return (int)(v < Tmax ? v : Tmax);
+}
+
+int pick_splits(int B, int Tmax, int Hkv, const cowa_params_t* p) {
+  const int hg = p->hkv_global > 0 ? p->hkv_global : Hkv;
+  const int vmax = max_visible(Tmax, hg, p);
+  // enough blocks to fill 148 SMs several times over, and splits short enough for shared memory
+  int by_fill = (148 * 16 + B * Hkv - 1) / (B * Hkv);
+  int by_cap = (vmax + (kChunkCap - 16) - 1) / (kChunkCap - 16);
+  int by_len = (vmax + 127) / 128;  // no point in splits shorter than 128 rows
+  int s = by_fill < by_len ? by_fill : by_len;
+  if (s < by_cap) s = by_cap;
+  return s < 1 ? 1 : s;
+}
+
+template <int D, int G>
+cudaError_t launch_split(const DecodeArgs& a, cudaStream_t st) {
+  dim3 grid(a.S, a.Hkv, a.B);
+  cowa_decode_split_kernel<D, G><<<grid, kThreads, 0, st>>>(a);
+  return cudaGetLastError();
+}
+
+template <int D>
+cudaError_t dispatch_split(int G, const DecodeArgs& a, cudaStream_t st) {
+  switch (G) {
+    case 1: return launch_split<D, 1>(a, st);
+    case 2: return launch_split<D, 2>(a, st);
+    case 4: return launch_split<D, 4>(a, st);
+    case 8: return launch_split<D, 8>(a, st);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+}  // namespace
+
+namespace cowa {
+
+// Validates a decode call; on success fills S (number of splits).
+int decode_validate(const void* q, const void* kc, const void* vc, const int32_t* lens, void* o, int B,
+                    int Tmax, int Hq, int Hkv, int D, const cowa_params_t* p, int* S) {
+  if (!q || !kc || !vc || !lens || !o || !p) return COWA_ERR_INVALID_ARG;
+  if (B <= 0 || Tmax <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0) return COWA_ERR_INVALID_ARG;
+  if (!p->full_attn && (p->sink < 0 || p->local < 1)) return COWA_ERR_INVALID_ARG;
+  const int hg = p->hkv_global > 0 ? p->hkv_global : Hkv;
+  if (p->hkv_offset < 0 || p->hkv_offset + Hkv > hg) return COWA_ERR_INVALID_ARG;
+  if (D != 64 && D != 128) return COWA_ERR_UNSUPPORTED;
+  const int G = Hq / Hkv;
+  if (G != 1 && G != 2 && G != 4 && G != 8) return COWA_ERR_UNSUPPORTED;
+  if (B > 65535 || Hkv > 65535) return COWA_ERR_UNSUPPORTED;
+  if (!aligned16(q) || !aligned16(kc) || !aligned16(vc) || !aligned16(o)) return COWA_ERR_MISALIGNED;
+  *S = pick_splits(B, Tmax, Hkv, p);
+  return COWA_OK;
+}
+
+size_t decode_ws_bytes(int B, int Hq, int D, int S) {
+  return (size_t)B * Hq * S * (D + 2) * sizeof(float);
+}
+
+// Enqueues the split and combine kernels using `ws` (>= decode_ws_bytes) as scratch.
+int decode_launch(const void* q, const void* kc, const void* vc, const int32_t* lens, void* o, float* lse,
+                  int B, int Tmax, int Hq, int Hkv, int D, const cowa_params_t* p, int S, void* ws,
+                  cudaStream_t st) {
+  DecodeArgs a;
+  a.q = static_cast<const __nv_bfloat16*>(q);
+  a.kc = static_cast<const __nv_bfloat16*>(kc);
+  a.vc = static_cast<const __nv_bfloat16*>(vc);
+  a.lens = lens;
+  a.ws_o = static_cast<float*>(ws);
+  a.ws_m = a.ws_o + (size_t)B * Hq * S * D;
+  a.ws_l = a.ws_m + (size_t)B * Hq * S;
+  a.B = B; a.Tmax = Tmax; a.Hq = Hq; a.Hkv = Hkv; a.S = S;
+  a.sink = p->sink; a.near = p->local;
+  a.hkv_global = p->hkv_global > 0 ? p->hkv_global : Hkv;
+  a.hkv_offset = p->hkv_offset;
+  a.full_attn = p->full_attn;
+  a.scale_log2 = p->softmax_scale * 1.4426950408889634f;
+  const int G = Hq / Hkv;
+  cudaError_t e = (D == 128) ? dispatch_split<128>(G, a, st) : dispatch_split<64>(G, a, st);
+  if (e != cudaSuccess) return record_cuda_error(e);
+  if (D == 128)
+    cowa_decode_combine_kernel<128><<<B * Hq, 128, 0, st>>>(a.ws_o, a.ws_m, a.ws_l,
+                                                            static_cast<__nv_bfloat16*>(o), lse, S);
+  else
+    cowa_decode_combine_kernel<64><<<B * Hq, 64, 0, st>>>(a.ws_o, a.ws_m, a.ws_l,
+                                                          static_cast<__nv_bfloat16*>(o), lse, S);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return record_cuda_error(e);
+  return COWA_OK;
+}
+
+}  // namespace cowa
+
+extern "C" {
+
+size_t cowa_decode_workspace_bytes(int B, int Tmax, int Hq, int Hkv, int D, const cowa_params_t* p) {
+  if (!p || B <= 0 || Tmax <= 0 || Hq <= 0 || Hkv <= 0 || D <= 0) return 0;
+  return cowa::decode_ws_bytes(B, Hq, D, pick_splits(B, Tmax, Hkv, p));
+}
+
+int cowa_decode(const void* q, const void* kcache, const void* vcache, const int32_t* lens, void* o,
+                float* lse, int B, int Tmax, int Hq, int Hkv, int D, const cowa_params_t* p,
+                void* workspace, size_t workspace_bytes, void* stream) {
+  int S = 0;
+  int st = cowa::decode_validate(q, kcache, vcache, lens, o, B, Tmax, Hq, Hkv, D, p, &S);
+  if (st != COWA_OK) return st;
+  if (!workspace) return COWA_ERR_INVALID_ARG;
+  if (!cowa::aligned16(workspace)) return COWA_ERR_MISALIGNED;
+  if (workspace_bytes < cowa::decode_ws_bytes(B, Hq, D, S)) return COWA_ERR_WORKSPACE_TOO_SMALL;
+  return cowa::decode_launch(q, kcache, vcache, lens, o, lse, B, Tmax, Hq, Hkv, D, p, S, workspace,
+                             static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

@@ -1,0 +1,338 @@
+// CoWindow Attention forward (Algorithm 1) for sm_100a.
+//
+// One thread block = one (batch, QO head, 128-row QO tile).  The block walks the tile's visited
+// KV tiles J_h(i) (analytic scheduler, descending order), and for each:
+//   TMA loads K / V tiles (128B-swizzled) -> tcgen05.mma S = Q K^T into TMEM -> each of the 128
+//   threads owns one row: tcgen05.ld, (boundary tiles only) window/causal mask from a per-row
+//   bit mask, online softmax in base 2 with the scale folded in, P written back to TMEM as
+//   bf16 over S's columns -> tcgen05.mma O += P V with P as the TMEM operand.
+// The running max is only advanced when the row max grows by more than 2^8 (the accumulator is
+// rescaled in TMEM only then); the final normalisation uses the same reference max, so the
+// result is the exact softmax.  Two blocks fit per SM (96 KB shared memory, 256 TMEM columns
+// each), which overlaps one block's softmax with the other's MMAs.  The 4 QO heads of a GQA
+// group at the same tile are adjacent in launch order and share K/V through L2.
+#include <cuda_bf16.h>
+
+#include "cowa_common.h"
+#include "cowa_ptx.cuh"
+#include "cowa_tma.h"
+
+using namespace cowa_ptx;
+
+namespace {
+
+constexpr int BQ = 128, BK = 128;
+
+struct FwdArgs {
+  float* lse;
+  unsigned int* status;
+  int B, Nq, Nk, Hq, Hkv, G;
+  float scale_log2;
+  CowaHeadWindows wins;
+};
+
+// bits [lo, hi] of the 32-bit word covering columns [base, base+32)
+__device__ __forceinline__ uint32_t interval_bits(int a, int b, int base) {
+  int lo = max(a - base, 0), hi = min(b - base, 31);
+  if (lo > hi) return 0u;
+  return (0xFFFFFFFFu >> (31 - (hi - lo))) << lo;
+}
+
+template <int D>
+struct FwdSmem {
+  static constexpr int kTile = 128 * D * 2;  // bytes of one 128-row tile
+  static constexpr int kQ = 0, kK = kTile, kV = 2 * kTile, kBar = 3 * kTile;
+  static constexpr int kBytes = 3 * kTile + 64 + 1024;  // + barriers + alignment slack
+};
+
+template <int D>
+__global__ void __launch_bounds__(128, 2)
+cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
+                const __grid_constant__ FwdArgs a) {
+  constexpr int NSLAB = D / 64;          // 64-element (128-byte) slabs along D
+  constexpr int SLAB = 128 * 128;        // bytes of one slab: 128 rows x 128 B
+  constexpr uint32_t TMEM_COLS = 256;    // S/P: [0,128), O: [128, 128+D)
+  constexpr uint32_t IDESC_S = idesc_bf16(128, BK, 0, 0);
+  constexpr uint32_t IDESC_O = idesc_bf16(128, D, 0, 1);
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sQ = smem + FwdSmem<D>::kQ;
+  uint8_t* sK = smem + FwdSmem<D>::kK;
+  uint8_t* sV = smem + FwdSmem<D>::kV;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + FwdSmem<D>::kBar);
+  uint64_t* bar_q = bars + 0;
+  uint64_t* bar_k = bars + 1;
+  uint64_t* bar_v = bars + 2;
+  uint64_t* bar_mma = bars + 3;
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 4);
+
+  const int tid = threadIdx.x, warp = tid >> 5;
+
+  // ---- work item (heaviest QO tiles first; the group's heads adjacent) ----
+  int idx = blockIdx.x;
+  const int g = idx % a.G; idx /= a.G;
+  const int hk = idx % a.Hkv; idx /= a.Hkv;
+  const int b = idx % a.B; idx /= a.B;
+  const int nQ = (a.Nq + BQ - 1) / BQ;
+  const int i = nQ - 1 - idx;
+  const int h = hk * a.G + g;
+  const int off = a.Nk - a.Nq;
+  const int q0 = i * BQ, q1 = min(q0 + BQ, a.Nq) - 1;
+  const CowaWin w = a.wins.w[hk];
+  CowaRange rg[3];
+  cowa_fwd_ranges(w, q0, q1, off, a.Nk, BK, rg);
+  const int ntiles = cowa_range_len(rg[0]) + cowa_range_len(rg[1]) + cowa_range_len(rg[2]);
+  const int bhq = b * a.Hq + h, bhk = b * a.Hkv + hk;
+
+  // ---- set-up ----
+  if (tid == 0) {
+    mbar_init(bar_q, 1); mbar_init(bar_k, 1); mbar_init(bar_v, 1); mbar_init(bar_mma, 1);
+    fence_mbar_init();
+    prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV); prefetch_tmap(&tmO);
+  }
+  if (warp == 0) {
+    __syncwarp();
+    tmem_alloc(tmem_holder, TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+  const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);  // this warp's 32 lanes
+  const uint32_t t_S = t_lane, t_O = t_lane + 128;
+
+  bool ok = true;  // false once a bounded wait ran out
+  uint32_t ph_k = 0, ph_v = 0, ph_mma = 0;
+
+  if (tid == 0 && ntiles > 0) {
+    const int j0 = cowa_fwd_tile_at(rg, 0);
+    mbar_expect_tx(bar_q, FwdSmem<D>::kTile);
+    for (int s = 0; s < NSLAB; ++s) tma_load_3d(sQ + s * SLAB, &tmQ, bar_q, s * 64, q0, bhq);
+    mbar_expect_tx(bar_k, FwdSmem<D>::kTile);
+    for (int s = 0; s < NSLAB; ++s) tma_load_3d(sK + s * SLAB, &tmK, bar_k, s * 64, j0 * BK, bhk);
+    mbar_expect_tx(bar_v, FwdSmem<D>::kTile);
+    for (int s = 0; s < NSLAB; ++s) tma_load_3d(sV + s * SLAB, &tmV, bar_v, s * 64, j0 * BK, bhk);
+  }
+
+  // ---- per-row state ----
+  const int row = q0 + tid;
+  const bool row_valid = row < a.Nq;
+  const int rowpos = row + off;  // position of this query on the key axis
+  float m_ref = -INFINITY, l_sum = 0.f;
+
+  for (int t = 0; t < ntiles; ++t) {
+    const int j = cowa_fwd_tile_at(rg, t);
+    const int k0 = j * BK;
+    const bool full = cowa_tile_full(w, q0, BQ, k0, BK, off, a.Nq, a.Nk);
+
+    // Thread 0 never leaves the loop on its own: a failed wait only clears `ok`, and every
+    // thread leaves together at the block-wide vote below.
+    if (tid == 0) {
+      if (t == 0) ok = ok && mbar_wait(bar_q, 0, a.status);
+      ok = ok && mbar_wait(bar_k, ph_k, a.status);
+      ph_k ^= 1;
+      if (ok) {
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t o = (kk / 4) * SLAB + (kk % 4) * 32;
+          mma_ss(tmem_base, smem_desc_sw128(smem_u32(sQ) + o, 16, 1024), smem_desc_sw128(smem_u32(sK) + o, 16, 1024),
+                 IDESC_S, kk > 0);
+        }
+      }
+      mma_commit(bar_mma);
+    }
+    __syncwarp();
+    ok = mbar_wait(bar_mma, ph_mma, a.status) && ok;
+    ph_mma ^= 1;
+    ok = __syncthreads_and(ok);
+    if (!ok) break;
+    tc_fence_after();
+
+    if (tid == 0) {  // S(t) is in TMEM, PV(t-1) is complete: both operand buffers are free again
+      if (t + 1 < ntiles) {
+        const int jn = cowa_fwd_tile_at(rg, t + 1);
+        mbar_expect_tx(bar_k, FwdSmem<D>::kTile);
+        for (int s = 0; s < NSLAB; ++s) tma_load_3d(sK + s * SLAB, &tmK, bar_k, s * 64, jn * BK, bhk);
+      }
+      if (t >= 1) {
+        mbar_expect_tx(bar_v, FwdSmem<D>::kTile);
+        for (int s = 0; s < NSLAB; ++s) tma_load_3d(sV + s * SLAB, &tmV, bar_v, s * 64, k0, bhk);
+      }
+    }
+    __syncwarp();
+
+    // ---- this thread's row of S ----
+    uint32_t sr[4][32];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) tmem_ld32(t_S + c * 32, sr[c]);
+    tmem_wait_ld();
+
+    uint32_t mask[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};
+    if (!full) {
+      const int kend = min(rowpos, a.Nk - 1);  // last causal key of this row
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const int base = k0 + c * 32;
+        uint32_t mk = interval_bits(rowpos - w.n + 1, kend, base) | interval_bits(0, min(w.s - 1, kend), base);
+        if (w.l > 0) mk |= interval_bits(rowpos - (w.n + w.g + w.l) + 1, min(rowpos - (w.n + w.g), kend), base);
+        mask[c] = row_valid ? mk : 0u;
+      }
+    }
+    float mx = -INFINITY;
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+#pragma unroll
+      for (int e = 0; e < 32; ++e) {
+        float s = __uint_as_float(sr[c][e]);
+        if (!full) s = (mask[c] >> e) & 1u ? s : -INFINITY;
+        sr[c][e] = __float_as_uint(s);
+        mx = fmaxf(mx, s);
+      }
+    mx *= a.scale_log2;
+    float m_new = m_ref;
+    if (mx > m_ref + 8.f) m_new = mx;
+    const float alpha = (m_new == m_ref) ? 1.f : ex2(m_ref - m_new);
+    const float sub = (m_new == -INFINITY) ? 0.f : m_new;
+    m_ref = m_new;
+
+    float rs = 0.f;
+    uint32_t pk[64];
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+#pragma unroll
+      for (int e = 0; e < 32; e += 2) {
+        const float p0 = ex2(fmaf(__uint_as_float(sr[c][e]), a.scale_log2, -sub));
+        const float p1 = ex2(fmaf(__uint_as_float(sr[c][e + 1]), a.scale_log2, -sub));
+        rs += p0 + p1;
+        pk[c * 16 + e / 2] = pack_bf16(p0, p1);
+      }
+    l_sum = l_sum * alpha + rs;
+
+    // P over S's first 64 columns
+#pragma unroll
+    for (int c = 0; c < 4; ++c) tmem_st16(t_S + c * 16, &pk[c * 16]);
+
+    // rescale the accumulator when some row of this warp moved its reference max
+    if (t > 0 && __any_sync(0xFFFFFFFFu, alpha != 1.f)) {
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t ov[32];
+        tmem_ld32(t_O + c * 32, ov);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 32; ++e) ov[e] = __float_as_uint(__uint_as_float(ov[e]) * alpha);
+        tmem_st32(t_O + c * 32, ov);
+      }
+    }
+    tmem_wait_st();
+    tc_fence_before();
+    __syncthreads();
+
+    if (tid == 0) {
+      ok = ok && mbar_wait(bar_v, ph_v, a.status);
+      ph_v ^= 1;
+      if (ok) {
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < BK / 16; ++kk) {
+          mma_ts(tmem_base + 128, tmem_base + kk * 8, smem_desc_sw128(smem_u32(sV) + kk * 2048, SLAB, 1024), IDESC_O,
+                 (t > 0 || kk > 0) ? 1u : 0u);
+        }
+      }
+      if (t == ntiles - 1) mma_commit(bar_mma);
+    }
+    __syncwarp();
+  }
+
+  // ---- epilogue: O / l, LSE ----
+  if (ntiles > 0) {
+    ok = mbar_wait(bar_mma, ph_mma, a.status) && ok;
+    ok = __syncthreads_and(ok);
+  }
+  if (ok && ntiles > 0) {
+    tc_fence_after();
+    const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
+#pragma unroll
+    for (int c = 0; c < D / 32; ++c) {
+      uint32_t ov[32];
+      tmem_ld32(t_O + c * 32, ov);
+      tmem_wait_ld();
+      // 32 columns = 4 chunks of 8 elements (16 B); slab = (c*32)/64, chunk index within slab
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        uint4 v;
+        v.x = pack_bf16(__uint_as_float(ov[q * 8 + 0]) * inv, __uint_as_float(ov[q * 8 + 1]) * inv);
+        v.y = pack_bf16(__uint_as_float(ov[q * 8 + 2]) * inv, __uint_as_float(ov[q * 8 + 3]) * inv);
+        v.z = pack_bf16(__uint_as_float(ov[q * 8 + 4]) * inv, __uint_as_float(ov[q * 8 + 5]) * inv);
+        v.w = pack_bf16(__uint_as_float(ov[q * 8 + 6]) * inv, __uint_as_float(ov[q * 8 + 7]) * inv);
+        const int d0 = c * 32 + q * 8;
+        const int slab = d0 / 64, chunk = (d0 % 64) / 8;
+        *reinterpret_cast<uint4*>(sQ + slab * SLAB + tid * 128 + ((chunk ^ (tid & 7)) << 4)) = v;
+      }
+    }
+    if (row_valid)
+      a.lse[(size_t)bhq * a.Nq + row] = 0.6931471805599453f * (m_ref + log2f(l_sum));
+    fence_proxy_async_smem();
+    __syncthreads();
+    if (tid == 0) {
+      for (int s = 0; s < NSLAB; ++s) tma_store_3d(&tmO, sQ + s * SLAB, s * 64, q0, bhq);
+      tma_commit_group();
+      tma_wait_group<0>();
+    }
+  }
+
+  // ---- teardown ----
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    __syncwarp();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+template <int D>
+int launch_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int T, int Hq, int Hkv,
+               const cowa_params_t* p, const CowaHeadWindows& hw, cudaStream_t st) {
+  CUtensorMap mq, mk, mv, mo;
+  int rc;
+  if ((rc = cowa::make_tensor_map_3d(&mq, q, cowa::MapType::BF16, D, T, (long long)B * Hq, 64, BQ))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mk, k, cowa::MapType::BF16, D, T, (long long)B * Hkv, 64, BK))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mv, v, cowa::MapType::BF16, D, T, (long long)B * Hkv, 64, BK))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mo, o, cowa::MapType::BF16, D, T, (long long)B * Hq, 64, BQ))) return rc;
+  FwdArgs a;
+  a.lse = lse;
+  a.status = cowa::device_status_word();
+  if (!a.status) return COWA_ERR_CUDA;
+  a.B = B; a.Nq = T; a.Nk = T; a.Hq = Hq; a.Hkv = Hkv; a.G = Hq / Hkv;
+  a.scale_log2 = p->softmax_scale * 1.4426950408889634f;
+  a.wins = hw;
+  COWA_CUDA_TRY(cudaFuncSetAttribute(cowa_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     FwdSmem<D>::kBytes));
+  const long long nblocks = (long long)((T + BQ - 1) / BQ) * B * Hq;
+  if (nblocks > 0x7FFFFFFFll) return COWA_ERR_UNSUPPORTED;
+  cowa_fwd_kernel<D><<<(unsigned)nblocks, 128, FwdSmem<D>::kBytes, st>>>(mq, mk, mv, mo, a);
+  COWA_CUDA_TRY(cudaGetLastError());
+  return COWA_OK;
+}
+
+}  // namespace
+
+extern "C" int cowa_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int T, int Hq,
+                        int Hkv, int D, const cowa_params_t* p, void* stream) {
+  if (!q || !k || !v || !o || !lse || !p) return COWA_ERR_INVALID_ARG;
+  if (B <= 0 || T <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0) return COWA_ERR_INVALID_ARG;
+  if (!(p->softmax_scale > 0.f)) return COWA_ERR_INVALID_ARG;
+  if (D != 64 && D != 128) return COWA_ERR_UNSUPPORTED;
+  if (!cowa::aligned16(q) || !cowa::aligned16(k) || !cowa::aligned16(v) || !cowa::aligned16(o))
+    return COWA_ERR_MISALIGNED;
+  CowaHeadWindows hw;
+  int rc = cowa::resolve_windows(T, Hkv, p, &hw);
+  if (rc != COWA_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  return D == 128 ? launch_fwd<128>(q, k, v, o, lse, B, T, Hq, Hkv, p, hw, st)
+                  : launch_fwd<64>(q, k, v, o, lse, B, T, Hq, Hkv, p, hw, st);
+}

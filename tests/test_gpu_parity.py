@@ -1,0 +1,186 @@
+"""GPU parity: the CUDA path (through the C ABI) against the float64 CPU oracle on the same
+seeded bf16 inputs.  Tolerances (bf16 inputs/outputs, fp32 accumulation, P rounded to bf16
+before its second product): O and gradients max-abs 2e-2 and mean-abs 2e-3, LSE max-abs 1e-3."""
+import numpy as np
+import pytest
+import torch
+
+import cowa_inputs
+import paper_2609_32704_b200 as cowa
+from oracle import cowa_oracle as orc
+
+pytestmark = pytest.mark.gpu
+
+TOL_MAX, TOL_MEAN, TOL_LSE = 2e-2, 2e-3, 1e-3
+DEV = "cuda"
+
+
+def check(name, got, want, tol_max=TOL_MAX, tol_mean=TOL_MEAN):
+    got = np.asarray(got, dtype=np.float64)
+    err = np.abs(got - want)
+    assert np.isfinite(got).all(), f"{name}: non-finite output"
+    assert err.max() <= tol_max, f"{name}: max-abs {err.max():.3e} > {tol_max}"
+    assert err.mean() <= tol_mean, f"{name}: mean-abs {err.mean():.3e} > {tol_mean}"
+
+
+def run_fwd(q, k, v, params):
+    B, Hq, T, D = q.shape
+    o = torch.full_like(q, float("nan"))
+    lse = torch.full((B, Hq, T), float("nan"), dtype=torch.float32, device=q.device)
+    cowa.cowa_fwd(q, k, v, o, lse, params)
+    torch.cuda.synchronize()
+    cowa.cowa_check_device_status()
+    return o, lse
+
+
+def fwd_case(B, T, Hq, Hkv, D, sink, local, seed=50, windows=None, full_attn=False):
+    q, k, v, _ = cowa_inputs.make_train_inputs(seed, B, T, Hq, Hkv, D)
+    scale = cowa_inputs.softmax_scale(D)
+    params = cowa.make_params(sink=sink, local=local, softmax_scale=scale, windows=windows, full_attn=full_attn)
+    o, lse = run_fwd(q.to(DEV), k.to(DEV), v.to(DEV), params)
+    if full_attn:
+        ws = [(0, T, 0, 0)] * Hkv
+    else:
+        ws = windows if windows is not None else orc.default_windows(T, Hkv, sink, local)
+    for b in range(B):
+        o_ref, lse_ref = orc.forward(cowa_inputs.to_f64(q[b]), cowa_inputs.to_f64(k[b]), cowa_inputs.to_f64(v[b]),
+                                     ws, scale)
+        check(f"lse[b={b}]", lse[b].cpu().numpy(), lse_ref, TOL_LSE, TOL_LSE)
+        check(f"o[b={b}]", o[b].float().cpu().numpy(), o_ref)
+
+
+# ------------------------------------------------------------------ forward
+
+def test_fwd_tiny_config():
+    c = cowa_inputs.CONFIGS["tiny"]
+    fwd_case(c["B"], c["T"], c["Hq"], c["Hkv"], c["D"], c["sink"], c["local"], seed=c["index"])
+
+
+@pytest.mark.parametrize("B,T,Hq,Hkv,D,sink,local", [
+    (1, 128, 1, 1, 128, 0, 128),      # one tile, dense
+    (1, 256, 2, 1, 128, 0, 1),        # near = 1: every row sees only itself (+ bands)
+    (2, 640, 8, 2, 128, 16, 100),     # bands not tile aligned
+    (1, 1000, 4, 4, 64, 7, 33),       # ragged tail, G = 1, D = 64
+    (1, 1100, 8, 1, 128, 5, 9),       # H_k = 1: dense causal through the bands
+    (1, 512, 4, 2, 128, 300, 300),    # sink + near > T: dense causal
+    (1, 1536, 16, 2, 64, 200, 64),    # G = 8, wide sink
+    (1, 77, 2, 2, 128, 3, 4),         # shorter than one tile
+])
+def test_fwd_shapes(B, T, Hq, Hkv, D, sink, local):
+    fwd_case(B, T, Hq, Hkv, D, sink, local)
+
+
+def test_fwd_full_attn_and_explicit_windows():
+    fwd_case(1, 900, 4, 2, 128, 0, 1, full_attn=True)
+    # duplicated-window control (both heads get the band nearest the near window) and a
+    # head-specific layout with a gap and no sink
+    ws = orc.duplicated_windows(1024, 2, 64, 128, 1)
+    fwd_case(1, 1024, 4, 2, 64, 64, 128, windows=ws)
+    fwd_case(1, 700, 2, 2, 128, 0, 1, windows=[(0, 50, 100, 200), (20, 10, 0, 0)])
+
+
+def test_fwd_8k_config_sampled_heads():
+    c = cowa_inputs.CONFIGS["8k"]
+    B, T, Hq, Hkv, D = c["B"], c["T"], c["Hq"], c["Hkv"], c["D"]
+    q, k, v, _ = cowa_inputs.make_train_inputs(c["index"], B, T, Hq, Hkv, D)
+    scale = cowa_inputs.softmax_scale(D)
+    params = cowa.make_params(sink=c["sink"], local=c["local"], softmax_scale=scale)
+    o, lse = run_fwd(q.to(DEV), k.to(DEV), v.to(DEV), params)
+    ws = orc.default_windows(T, Hkv, c["sink"], c["local"])
+    rows = np.arange(T)
+    for b, h in [(0, 0), (0, 7), (1, 9), (1, 15)]:
+        o_ref, lse_ref = orc.forward_rows(cowa_inputs.to_f64(q[b]), cowa_inputs.to_f64(k[b]),
+                                          cowa_inputs.to_f64(v[b]), ws, scale, h, rows)
+        check(f"lse[{b},{h}]", lse[b, h].cpu().numpy(), lse_ref, TOL_LSE, TOL_LSE)
+        check(f"o[{b},{h}]", o[b, h].float().cpu().numpy(), o_ref)
+    # duplicated-window control at the same shape: one head pair
+    wd = orc.duplicated_windows(T, Hkv, c["sink"], c["local"], 1)
+    pd = cowa.make_params(softmax_scale=scale, windows=wd)
+    o, lse = run_fwd(q.to(DEV), k.to(DEV), v.to(DEV), pd)
+    o_ref, lse_ref = orc.forward_rows(cowa_inputs.to_f64(q[0]), cowa_inputs.to_f64(k[0]), cowa_inputs.to_f64(v[0]),
+                                      wd, scale, 13, rows)
+    check("dup lse", lse[0, 13].cpu().numpy(), lse_ref, TOL_LSE, TOL_LSE)
+    check("dup o", o[0, 13].float().cpu().numpy(), o_ref)
+
+
+# ------------------------------------------------------------------ decode
+
+def run_decode(q, kc, vc, lens, params):
+    B, Hq, D = q.shape
+    Hkv, Tmax = kc.shape[1], kc.shape[2]
+    o = torch.full_like(q, float("nan"))
+    lse = torch.full((B, Hq), float("nan"), dtype=torch.float32, device=q.device)
+    nbytes = cowa.cowa_decode_workspace_bytes(B, Tmax, Hq, Hkv, D, params)
+    ws = torch.empty(nbytes + 64, dtype=torch.uint8, device=q.device)
+    ws.fill_(0xFF)  # NaN pattern: the workspace needs no initialisation
+    cowa.cowa_decode(q, kc, vc, lens, o, lse, params, ws[:nbytes])
+    torch.cuda.synchronize()
+    assert (ws[nbytes:] == 0xFF).all(), "decode wrote past its workspace"
+    return o, lse
+
+
+def decode_case(B, Tmax, Hq, Hkv, D, sink, local, lens, seed=60, full_attn=False):
+    q, kc, vc, _ = cowa_inputs.make_decode_inputs(seed, B, Tmax, Hq, Hkv, D, Tmax, Tmax)
+    lens = torch.tensor(lens, dtype=torch.int32)
+    for b in range(B):  # NaN beyond the chosen lengths: an over-read shows up
+        kc[b, :, int(lens[b]):] = float("nan")
+        vc[b, :, int(lens[b]):] = float("nan")
+    scale = cowa_inputs.softmax_scale(D)
+    params = cowa.make_params(sink=sink, local=local, softmax_scale=scale, full_attn=full_attn)
+    o, lse = run_decode(q.to(DEV), kc.to(DEV), vc.to(DEV), lens.to(DEV), params)
+    if full_attn:
+        sink, local = 0, Tmax
+    kf, vf = kc.float().numpy(), vc.float().numpy()
+    o_ref, lse_ref = orc.decode(cowa_inputs.to_f64(q), kf, vf, lens.numpy(), sink, local, scale)
+    check("decode lse", lse.cpu().numpy(), lse_ref, TOL_LSE, TOL_LSE)
+    check("decode o", o.float().cpu().numpy(), o_ref)
+
+
+@pytest.mark.parametrize("B,Tmax,Hq,Hkv,D,sink,local,lens", [
+    (3, 5000, 8, 2, 128, 16, 100, [5000, 1, 2777]),
+    (2, 3001, 8, 8, 64, 4, 31, [3001, 17]),            # G = 1, D = 64
+    (2, 4096, 16, 2, 128, 128, 512, [4096, 640]),      # G = 8; second sequence is dense
+    (1, 40000, 4, 2, 128, 128, 4096, [39999]),         # several splits per head
+    (4, 300, 4, 2, 64, 0, 5, [300, 299, 6, 5]),        # no sink
+])
+def test_decode_shapes(B, Tmax, Hq, Hkv, D, sink, local, lens):
+    decode_case(B, Tmax, Hq, Hkv, D, sink, local, lens)
+
+
+def test_decode_full_attn():
+    decode_case(2, 9000, 8, 2, 128, 0, 1, [9000, 4321], full_attn=True)
+
+
+def test_decode_128k_config():
+    c = cowa_inputs.CONFIGS["decode128k"]
+    q, kc, vc, lens = cowa_inputs.make_decode_inputs(c["index"], c["B"], c["Tmax"], c["Hq"], c["Hkv"], c["D"],
+                                                     c["len_lo"], c["len_hi"], device=DEV)
+    scale = cowa_inputs.softmax_scale(c["D"])
+    params = cowa.make_params(sink=c["sink"], local=c["local"], softmax_scale=scale)
+    o, lse = run_decode(q, kc, vc, lens, params)
+    lens_h = lens.cpu().numpy()
+    o_h, lse_h = o.float().cpu().numpy(), lse.cpu().numpy()
+    # the oracle walks each head's visible rows only; move one (sequence, KV head) at a time
+    G = c["Hq"] // c["Hkv"]
+    for b in range(c["B"]):
+        for hk in range(c["Hkv"]):
+            kf = kc[b:b + 1, hk:hk + 1].cpu().to(torch.float64).numpy()
+            vf = vc[b:b + 1, hk:hk + 1].cpu().to(torch.float64).numpy()
+            qf = q[b:b + 1, hk * G:(hk + 1) * G].cpu().to(torch.float64).numpy()
+            o_ref, lse_ref = orc.decode(qf, kf, vf, lens_h[b:b + 1], c["sink"], c["local"], scale,
+                                        h_k_global=c["Hkv"], hk_offset=hk)
+            check(f"decode lse[{b},{hk}]", lse_h[b, hk * G:(hk + 1) * G], lse_ref[0], TOL_LSE, TOL_LSE)
+            check(f"decode o[{b},{hk}]", o_h[b, hk * G:(hk + 1) * G], o_ref[0])
+
+
+def test_decode_equals_last_forward_row():
+    # cross-path: decode output == last row of the training forward at T = len
+    T, Hq, Hkv, D, sink, local = 1500, 4, 2, 128, 32, 200
+    q, k, v, _ = cowa_inputs.make_train_inputs(61, 1, T, Hq, Hkv, D, device=DEV)
+    scale = cowa_inputs.softmax_scale(D)
+    params = cowa.make_params(sink=sink, local=local, softmax_scale=scale)
+    o_f, lse_f = run_fwd(q, k, v, params)
+    lens = torch.tensor([T], dtype=torch.int32, device=DEV)
+    o_d, lse_d = run_decode(q[:, :, T - 1].contiguous(), k, v, lens, params)
+    assert (o_d.float() - o_f[:, :, T - 1].float()).abs().max().item() <= 2e-2
+    assert (lse_d - lse_f[:, :, T - 1]).abs().max().item() <= 1e-3
