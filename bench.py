@@ -1,0 +1,428 @@
+#!/usr/bin/env python
+"""Benchmark of the CoWA hot path on B200.
+
+One step = one pass of the whole hot path on seeded synthetic inputs:
+  training forward + backward at the 128K configuration (B=1, T=131072, Hq=32, Hkv=8, D=128,
+  sink 128, near 4096) followed by one split-KV decode step of the 128K decode configuration
+  (batch 8, lengths in [96K, 128K]).
+`value` is TFLOP/s over visited tiles of forward + backward (4*D resp. 10*D FLOPs per visited
+query-key pair and QO head); the decode phase is reported beside it (us per step, GB/s).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W]          # the CUDA library
+    python bench.py --impl reference [...]                       # the CPU oracle, bounded sample
+
+Under torchrun every rank runs the same workload on its own GPU (independent replicas: the
+operator has no exchange step); rank 0 prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+TRAIN_CFG, DECODE_CFG = "128k", "decode128k"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_setup(n_gpus):
+    import torch
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        torch.cuda.set_device(0)
+    return rank, world, local
+
+
+def barrier(world):
+    import torch
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.synchronize()
+
+
+def max_over_ranks(x, world):
+    import torch
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device="cuda")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+# ------------------------------------------------------------------------------------------
+# CPU oracle timing (bounded sample of the 128K forward), used by cpu_baseline and --impl reference
+# ------------------------------------------------------------------------------------------
+
+def oracle_sample(budget_s, seed_tiles=0):
+    """Times the oracle's forward on whole 128-row query tiles of the 128K configuration, one
+    (head, tile) at a time, until about budget_s seconds are spent.  Returns FLOPs over legal
+    pairs (4*D per pair) and the seconds used."""
+    import numpy as np
+    import torch
+    import cowa_inputs
+    from oracle import cowa_oracle as orc
+    c = cowa_inputs.CONFIGS[TRAIN_CFG]
+    T, Hq, Hkv, D = c["T"], c["Hq"], c["Hkv"], c["D"]
+    G = Hq // Hkv
+    ws = orc.default_windows(T, Hkv, c["sink"], c["local"])
+    scale = cowa_inputs.softmax_scale(D)
+    g = torch.Generator().manual_seed(c["index"] * 1000 + 7)
+    # one KV head's tensors (synthetic N(0,1), bf16-rounded like the GPU inputs), reused by every sample
+    flops, secs, units = 0.0, 0.0, 0
+    rng = np.random.default_rng(seed_tiles)
+    k = torch.randn(1, T, D, generator=g).to(torch.bfloat16).to(torch.float64).numpy()
+    v = torch.randn(1, T, D, generator=g).to(torch.bfloat16).to(torch.float64).numpy()
+    q = torch.randn(1, T, D, generator=g).to(torch.bfloat16).to(torch.float64).numpy()
+    while secs < budget_s:
+        hk = int(rng.integers(0, Hkv))
+        tile = int(rng.integers(0, T // 128))
+        rows = np.arange(tile * 128, tile * 128 + 128)
+        t0 = time.perf_counter()
+        orc.forward_rows(q, k, v, [ws[hk]], scale, 0, rows)
+        secs += time.perf_counter() - t0
+        pairs = int(orc.visible_mask(T, T, ws[hk], rows).sum())
+        flops += 4.0 * D * pairs
+        units += 1
+    return flops, secs, units
+
+
+def cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 0) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy  # noqa: F401  (loads BLAS so that the thread count can be read)
+    per_step = 6.0
+    for _ in range(args.warmup):
+        oracle_sample(0.5)
+    flops, secs = 0.0, 0.0
+    for s in range(args.steps):
+        f, t, _ = oracle_sample(per_step, seed_tiles=s)
+        flops, secs = flops + f, secs + t
+    val = flops / secs / 1e12
+    sample = (f"oracle forward on random (KV head, 128-row query tile) samples of the 128K configuration, "
+              f"~{per_step:.0f} s per step")
+    line = {
+        "impl": "reference", "metric": "cowa_train_tflops_visited_tiles_128k", "value": val, "unit": "TFLOP/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": TRAIN_CFG, "note": "float64 CPU oracle, legal-pair FLOPs of the sampled tiles"},
+        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cpu_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------
+# CUDA library
+# ------------------------------------------------------------------------------------------
+
+def run_cuda(args):
+    import torch
+    import cowa_inputs
+    import paper_2609_32704_b200 as cowa
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    rank, world, local = dist_setup(args.gpus)
+    dev = torch.device("cuda", torch.cuda.current_device())
+    peaks, peak_src = load_peaks()
+
+    ct = cowa_inputs.CONFIGS[TRAIN_CFG]
+    cd = cowa_inputs.CONFIGS[DECODE_CFG]
+    B, T, Hq, Hkv, D = ct["B"], ct["T"], ct["Hq"], ct["Hkv"], ct["D"]
+    scale = cowa_inputs.softmax_scale(D)
+    p_train = cowa.make_params(sink=ct["sink"], local=ct["local"], softmax_scale=scale)
+    p_full = cowa.make_params(softmax_scale=scale, full_attn=True)
+    p_dec = cowa.make_params(sink=cd["sink"], local=cd["local"], softmax_scale=scale)
+
+    # ---- inputs resident in HBM ----
+    q, k, v, d_o = cowa_inputs.make_train_inputs(ct["index"], B, T, Hq, Hkv, D, device=dev)
+    o = torch.empty_like(q)
+    lse = torch.empty((B, Hq, T), dtype=torch.float32, device=dev)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    ws_bwd = torch.empty(max(cowa.cowa_bwd_workspace_bytes(B, T, Hq, Hkv, D, p_train), 16), dtype=torch.uint8,
+                         device=dev)
+    qd, kc, vc, lens = cowa_inputs.make_decode_inputs(cd["index"], cd["B"], cd["Tmax"], cd["Hq"], cd["Hkv"], cd["D"],
+                                                      cd["len_lo"], cd["len_hi"], device=dev)
+    od = torch.empty_like(qd)
+    lsed = torch.empty((cd["B"], cd["Hq"]), dtype=torch.float32, device=dev)
+    ws_dec = torch.empty(cowa.cowa_decode_workspace_bytes(cd["B"], cd["Tmax"], cd["Hq"], cd["Hkv"], cd["D"], p_dec),
+                         dtype=torch.uint8, device=dev)
+
+    # ---- work counts ----
+    cnt = cowa.cowa_tile_counts(T, T, Hkv, p_train)
+    cnt_full = cowa.cowa_tile_counts(T, T, Hkv, p_full)
+    G = Hq // Hkv
+    fwd_flops = cnt["visited"] * 128 * 128 * 4 * D * G * B
+    bwd_flops = 2.5 * fwd_flops
+    full_fwd_flops = cnt_full["visited"] * 128 * 128 * 4 * D * G * B
+    lens_h = lens.cpu().tolist()
+    vis_rows = 0
+    for n in lens_h:
+        for w_ in cowa.cowa_default_windows(n, cd["Hkv"], 0, cd["Hkv"], cd["sink"], cd["local"]):
+            vis_rows += min(n, w_[0] + w_[1] + w_[3])
+    dec_bytes = vis_rows * cd["D"] * 2 * 2
+
+    have_bwd = True
+    try:
+        cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, p_train, ws_bwd)
+    except cowa.CowaError as e:
+        if e.status != -2:
+            raise
+        have_bwd = False
+    torch.cuda.synchronize()
+
+    def step(params, ev=None):
+        if ev: ev[0].record()
+        cowa.cowa_fwd(q, k, v, o, lse, params)
+        if ev: ev[1].record()
+        if have_bwd:
+            cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, params, ws_bwd)
+        if ev: ev[2].record()
+        cowa.cowa_decode(qd, kc, vc, lens, od, lsed, p_dec, ws_dec)
+        if ev: ev[3].record()
+
+    for _ in range(args.warmup):
+        step(p_train)
+    torch.cuda.synchronize()
+    cowa.cowa_check_device_status()
+
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    sampler = ClockSampler(torch.cuda.current_device())
+    if rank == 0:
+        sampler.start()
+    barrier(world)
+    for s in range(args.steps):
+        step(p_train, evs[s])
+    barrier(world)
+    clocks = sampler.stop() if rank == 0 else None
+    cowa.cowa_check_device_status()
+
+    fwd_ms = sum(e[0].elapsed_time(e[1]) for e in evs) / args.steps
+    bwd_ms = sum(e[1].elapsed_time(e[2]) for e in evs) / args.steps
+    dec_ms = sum(e[2].elapsed_time(e[3]) for e in evs) / args.steps
+    total_ms = evs[0][0].elapsed_time(evs[-1][3]) / args.steps
+    fwd_ms, bwd_ms, dec_ms, total_ms = (max_over_ranks(x, world) for x in (fwd_ms, bwd_ms, dec_ms, total_ms))
+
+    train_flops = fwd_flops + (bwd_flops if have_bwd else 0.0)
+    train_ms = fwd_ms + (bwd_ms if have_bwd else 0.0)
+    value = world * train_flops / (train_ms * 1e-3) / 1e12
+
+    # ---- FullAttn path of the same library (few iterations: it is ~5.4x the work) ----
+    full = {}
+    if rank == 0 and not args.no_fullattn:
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        cowa.cowa_fwd(q, k, v, o, lse, p_full)
+        torch.cuda.synchronize()
+        e[0].record()
+        cowa.cowa_fwd(q, k, v, o, lse, p_full)
+        e[1].record()
+        if have_bwd:
+            cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, p_full, ws_bwd)
+        e[2].record()
+        torch.cuda.synchronize()
+        f_ms, b_ms = e[0].elapsed_time(e[1]), e[1].elapsed_time(e[2])
+        full = {"fullattn_fwd_ms": f_ms, "fullattn_fwd_tflops": full_fwd_flops / f_ms / 1e9,
+                "speedup_fwd": f_ms / fwd_ms, "work_ratio_tiles": cnt_full["visited"] / cnt["visited"]}
+        if have_bwd:
+            full.update({"fullattn_bwd_ms": b_ms, "speedup_bwd": b_ms / bwd_ms})
+        # decode FullAttn: every head reads the whole prefix
+        ws_df = torch.empty(cowa.cowa_decode_workspace_bytes(cd["B"], cd["Tmax"], cd["Hq"], cd["Hkv"], cd["D"], p_full),
+                            dtype=torch.uint8, device=dev)
+        cowa.cowa_decode(qd, kc, vc, lens, od, lsed, p_full, ws_df)
+        torch.cuda.synchronize()
+        e2 = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        e2[0].record()
+        for _ in range(5):
+            cowa.cowa_decode(qd, kc, vc, lens, od, lsed, p_full, ws_df)
+        e2[1].record()
+        torch.cuda.synchronize()
+        fd_ms = e2[0].elapsed_time(e2[1]) / 5
+        full.update({"fullattn_decode_us": fd_ms * 1e3, "speedup_decode": fd_ms / dec_ms,
+                     "byte_ratio_decode": sum(lens_h) * cd["Hkv"] / vis_rows})
+        del ws_df
+
+    # ---- end to end: host buffers in, results back to the host, copies inside the timed region ----
+    e2e = None
+    if not args.no_e2e:
+        hq, hk_, hv, hdo = (x.cpu().pin_memory() for x in (q, k, v, d_o))
+        ho = torch.empty_like(hq).pin_memory()
+        hlse = torch.empty(lse.shape, dtype=torch.float32).pin_memory()
+        hdq, hdk, hdv = (torch.empty_like(x).pin_memory() for x in (hq, hk_, hv))
+        h2d = sum(x.numel() * x.element_size() for x in ((hq, hk_, hv, hdo) if have_bwd else (hq, hk_, hv)))
+        d2h = sum(x.numel() * x.element_size() for x in ((ho, hlse, hdq, hdk, hdv) if have_bwd else (ho, hlse)))
+
+        def e2e_step():
+            q.copy_(hq, non_blocking=True); k.copy_(hk_, non_blocking=True); v.copy_(hv, non_blocking=True)
+            cowa.cowa_fwd(q, k, v, o, lse, p_train)
+            ho.copy_(o, non_blocking=True); hlse.copy_(lse, non_blocking=True)
+            if have_bwd:
+                d_o.copy_(hdo, non_blocking=True)
+                cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, p_train, ws_bwd)
+                hdq.copy_(dq, non_blocking=True); hdk.copy_(dk, non_blocking=True); hdv.copy_(dv, non_blocking=True)
+
+        e2e_step()
+        barrier(world)
+        n_e2e = max(1, min(args.steps, 3))
+        ee = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        ee[0].record()
+        for _ in range(n_e2e):
+            e2e_step()
+        ee[1].record()
+        barrier(world)
+        e_ms = max_over_ranks(ee[0].elapsed_time(ee[1]) / n_e2e, world)
+        e2e = {"value": world * train_flops / (e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e_ms,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e}
+        del hq, hk_, hv, hdo, ho, hlse, hdq, hdk, hdv
+
+    if rank != 0:
+        return
+
+    # ---- roofline of the dominant kernel ----
+    if have_bwd and bwd_ms >= fwd_ms:
+        dom, dom_flops, dom_ms = "cowa_bwd main kernel", bwd_flops, bwd_ms
+    else:
+        dom, dom_flops, dom_ms = "cowa_fwd_kernel<128>", fwd_flops, fwd_ms
+    peak_tf = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+    achieved = dom_flops / dom_ms / 1e9
+    roofline = {"kernel": dom, "bound": "tensor", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s",
+                "frac": achieved / peak_tf, "peak_source": f"{peak_src} bf16 sustained (kernel timed inside a long step)",
+                "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "traffic": None}
+    dec_gbs = dec_bytes / (dec_ms * 1e-3) / 1e9
+    decode = {"us_per_step": dec_ms * 1e3, "us_per_token": dec_ms * 1e3 / cd["B"], "visible_kv_bytes": dec_bytes,
+              "achieved_gbs": dec_gbs, "hbm_peak_gbs": peaks["hbm_gbs"], "frac_hbm": dec_gbs / peaks["hbm_gbs"]}
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        f, t, units = oracle_sample(args.cpu_seconds)
+        cpu = {"value": f / t / 1e12, "unit": "TFLOP/s", "cores": cpu_threads(), "kind": "oracle",
+               "sample": f"oracle forward of {units} random (KV head, 128-row query tile) units of the 128K "
+                         f"configuration, {t:.1f} s; legal-pair FLOPs"}
+
+    line = {
+        "metric": "cowa_train_tflops_visited_tiles_128k", "value": value, "unit": "TFLOP/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": TRAIN_CFG, "decode_workload": DECODE_CFG, "B": B, "T": T, "Hq": Hq, "Hkv": Hkv,
+                   "D": D, "sink": ct["sink"], "near": ct["local"],
+                   "phases": ["fwd"] + (["bwd"] if have_bwd else []) + ["decode"],
+                   "l2": "inputs larger than L2 (2.6 GB training tensors, 0.57 GB visible KV cache)",
+                   "parallelism": "independent replicas" if world > 1 else "single GPU"},
+        "fwd_ms": fwd_ms, "fwd_tflops": fwd_flops / fwd_ms / 1e9,
+        "bwd_ms": bwd_ms if have_bwd else None, "bwd_tflops": bwd_flops / bwd_ms / 1e9 if have_bwd else None,
+        "visited_tiles": cnt["visited"], "causal_tiles": cnt["causal"],
+        "decode": decode, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
+        "gpu_launches": args.steps * (1 + (BWD_LAUNCHES if have_bwd else 0) + 2),
+    }
+    line.update(full)
+    print(json.dumps(line))
+
+
+BWD_LAUNCHES = 3  # preprocess, main kernel, dq conversion
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--no-fullattn", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        import torch.distributed as dist
+        if dist.is_initialized():
+            dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
