@@ -43,7 +43,8 @@ typedef enum {
   COWA_ERR_MISALIGNED = -3,         /* a base pointer is not 16-byte aligned */
   COWA_ERR_WORKSPACE_TOO_SMALL = -4,
   COWA_ERR_CUDA = -5,               /* a CUDA call failed; see cowa_last_cuda_error() */
-  COWA_ERR_DEVICE_TIMEOUT = -6      /* reported by cowa_check_device_status(): a bounded device wait ran out */
+  COWA_ERR_DEVICE_TIMEOUT = -6,     /* reported by cowa_check_device_status(): a bounded device wait ran out */
+  COWA_ERR_STATIC_SCRATCH_EXCEEDED = -7 /* cowa_decode_static: the call needs more scratch than the built-in array holds */
 } cowa_status_t;
 
 /* One KV head's windows: the paper's 4-tuple (sink width, near width, gap after the
@@ -93,6 +94,34 @@ int cowa_bwd(const void* q, const void* k, const void* v, const void* o, const f
 int cowa_decode(const void* q, const void* kcache, const void* vcache, const int32_t* lens,
                 void* o, float* lse, int B, int Tmax, int Hq, int Hkv, int D,
                 const cowa_params_t* p, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Decode for callers that cannot allocate device memory.  (No counterpart in the paper: this
+ * is a packaging variant of cowa_decode, same arguments minus the workspace, same results.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a serving loop that
+ * forbids allocation after start-up, in a plugin whose host owns all device memory, or in a
+ * region where an allocation's implicit synchronisation would stall other streams.  Such a
+ * caller cannot size and hand over the split-KV workspace that cowa_decode wants, so here the
+ * partial states go to a fixed array compiled into the library's device image instead
+ * (cowa_decode_static_capacity() bytes, 8 MiB; each GPU that loads the library holds that much
+ * until the process ends).  The call itself performs no cudaMalloc/cudaFree and calls nothing
+ * that allocates.
+ *
+ * Limits and rules:
+ *   - The call is rejected with COWA_ERR_STATIC_SCRATCH_EXCEEDED, before any launch, when
+ *     cowa_decode_workspace_bytes(...) for the same arguments exceeds the capacity
+ *     (for orientation: batch 8 x 32 QO heads x D 128 over a 128K cache needs 4.9 MiB).
+ *   - The first call on each device looks up the array's device address (one
+ *     cudaGetSymbolAddress with that device current).  Make that first call during set-up,
+ *     before any stream capture.
+ *   - All calls on a device share the one array.  It keeps the previous call's contents; that
+ *     is harmless because every value the merge kernel reads is rewritten by the same call's
+ *     split kernel first.  Two calls that overlap on the GPU (different streams, no ordering
+ *     between them) race on the array and give wrong results: serialise them. */
+int cowa_decode_static(const void* q, const void* kcache, const void* vcache, const int32_t* lens,
+                       void* o, float* lse, int B, int Tmax, int Hq, int Hkv, int D,
+                       const cowa_params_t* p, void* stream);
+size_t cowa_decode_static_capacity(void);
 
 size_t cowa_bwd_workspace_bytes(int B, int T, int Hq, int Hkv, int D, const cowa_params_t* p);
 size_t cowa_decode_workspace_bytes(int B, int Tmax, int Hq, int Hkv, int D, const cowa_params_t* p);

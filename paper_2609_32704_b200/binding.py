@@ -52,6 +52,10 @@ def lib():
         L.cowa_bwd.restype = i32
         L.cowa_decode.argtypes = [vp] * 6 + [i32] * 5 + [pp, vp, sz, vp]
         L.cowa_decode.restype = i32
+        L.cowa_decode_static.argtypes = [vp] * 6 + [i32] * 5 + [pp, vp]
+        L.cowa_decode_static.restype = i32
+        L.cowa_decode_static_capacity.argtypes = []
+        L.cowa_decode_static_capacity.restype = sz
         L.cowa_bwd_workspace_bytes.argtypes = [i32] * 5 + [pp]
         L.cowa_bwd_workspace_bytes.restype = sz
         L.cowa_decode_workspace_bytes.argtypes = [i32] * 5 + [pp]
@@ -155,6 +159,26 @@ def cowa_decode(q, kcache, vcache, lens, o, lse, params, workspace):
     _check(lib().cowa_decode(_ptr(q), _ptr(kcache), _ptr(vcache), _ptr(lens), _ptr(o), _ptr(lse), B, Tmax,
                              Hq, Hkv, D, C.byref(params), _ptr(workspace),
                              workspace.numel() * workspace.element_size(), _stream()), "cowa_decode")
+
+
+def cowa_decode_static_capacity():
+    return int(lib().cowa_decode_static_capacity())
+
+
+def cowa_decode_static(q, kcache, vcache, lens, o, lse, params):
+    """cowa_decode without a workspace argument: for callers that may not allocate device
+    memory.  The split states go to a fixed 8 MiB array inside the library; calls that need more
+    raise CowaError (status -7).  Calls that overlap on the GPU must be serialised."""
+    import torch
+    for t, n in ((q, "q"), (kcache, "kcache"), (vcache, "vcache"), (o, "o")):
+        _need(t, torch.bfloat16, n)
+    _need(lens, torch.int32, "lens")
+    if lse is not None:
+        _need(lse, torch.float32, "lse")
+    B, Hq, D = q.shape
+    Hkv, Tmax = kcache.shape[1], kcache.shape[2]
+    _check(lib().cowa_decode_static(_ptr(q), _ptr(kcache), _ptr(vcache), _ptr(lens), _ptr(o), _ptr(lse), B,
+                                    Tmax, Hq, Hkv, D, C.byref(params), _stream()), "cowa_decode_static")
 
 
 def cowa_default_windows(Nk, Hkv_global, hkv_offset, Hkv_local, sink, local):

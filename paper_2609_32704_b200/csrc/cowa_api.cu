@@ -181,6 +181,8 @@ const char* cowa_status_string(int status) {
     case COWA_ERR_WORKSPACE_TOO_SMALL: return "workspace or output buffer too small";
     case COWA_ERR_CUDA: return "CUDA call failed";
     case COWA_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+    case COWA_ERR_STATIC_SCRATCH_EXCEEDED:
+      return "cowa_decode_static: the call needs more scratch than the library's built-in array holds";
     default: return "unknown status";
   }
 }

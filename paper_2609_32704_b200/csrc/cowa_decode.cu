@@ -24,6 +24,29 @@ namespace {
 constexpr int kThreads = 128;
 constexpr int kChunkCap = 1024;  // max visible rows per split (scores of a split live in shared memory)
 
+// Scratch of cowa_decode_static: lives in the library's device image, so every GPU that loads the
+// library keeps these bytes reserved until the process exits.
+constexpr size_t kStaticScratchBytes = 8u << 20;
+static __device__ __align__(256) unsigned char g_decode_static_scratch[kStaticScratchBytes];
+
+// Device address of the scratch array on the current device.  The array's name is only a
+// host-side handle here; the address the kernels need comes from cudaGetSymbolAddress, looked
+// up once per device with that device current.
+void* static_scratch_ptr(cudaError_t* err) {
+  static void* cache[64] = {nullptr};
+  int dev = 0;
+  *err = cudaGetDevice(&dev);
+  if (*err != cudaSuccess) return nullptr;
+  if (dev < 0 || dev >= 64) { *err = cudaErrorInvalidDevice; return nullptr; }
+  if (!cache[dev]) {
+    void* ptr = nullptr;
+    *err = cudaGetSymbolAddress(&ptr, g_decode_static_scratch);
+    if (*err != cudaSuccess) return nullptr;
+    cache[dev] = ptr;
+  }
+  return cache[dev];
+}
+
 struct DecodeArgs {
   const __nv_bfloat16* q;
   const __nv_bfloat16* kc;
@@ -367,6 +390,24 @@ int cowa_decode(const void* q, const void* kcache, const void* vcache, const int
   if (!cowa::aligned16(workspace)) return COWA_ERR_MISALIGNED;
   if (workspace_bytes < cowa::decode_ws_bytes(B, Hq, D, S)) return COWA_ERR_WORKSPACE_TOO_SMALL;
   return cowa::decode_launch(q, kcache, vcache, lens, o, lse, B, Tmax, Hq, Hkv, D, p, S, workspace,
+                             static_cast<cudaStream_t>(stream));
+}
+
+size_t cowa_decode_static_capacity(void) { return kStaticScratchBytes; }
+
+int cowa_decode_static(const void* q, const void* kcache, const void* vcache, const int32_t* lens, void* o,
+                       float* lse, int B, int Tmax, int Hq, int Hkv, int D, const cowa_params_t* p,
+                       void* stream) {
+  int S = 0;
+  int st = cowa::decode_validate(q, kcache, vcache, lens, o, B, Tmax, Hq, Hkv, D, p, &S);
+  if (st != COWA_OK) return st;
+  if (cowa::decode_ws_bytes(B, Hq, D, S) > kStaticScratchBytes) return COWA_ERR_STATIC_SCRATCH_EXCEEDED;
+  cudaError_t e = cudaSuccess;
+  void* scratch = static_scratch_ptr(&e);
+  if (!scratch) return cowa::record_cuda_error(e);
+  // Every slot of the split states that the merge kernel reads is written by the split kernel of
+  // the same call, so nothing left over from an earlier call needs clearing.
+  return cowa::decode_launch(q, kcache, vcache, lens, o, lse, B, Tmax, Hq, Hkv, D, p, S, scratch,
                              static_cast<cudaStream_t>(stream));
 }
 
