@@ -1,20 +1,537 @@
-// CoWindow Attention backward (Algorithm 2) -- placeholder until the kernels land.
+// CoWindow Attention backward (Algorithm 2) for sm_100a.
+//
+// Three launches on the caller's stream:
+//   1. preprocess   Delta = rowsum(O * dO) (Algorithm 2 line 13) and LSE * log2(e), fp32 row vectors
+//                   padded to a multiple of 64 rows (padding: LSE = +inf, so that P = 0 there);
+//                   the fp32 dQ accumulator is zeroed by a memset before it.
+//   2. main kernel  one thread block per (batch, KV head, 128-row KV tile), KV-stationary as in
+//                   Algorithm 2, looping over the G QO heads of the group and over the 64-row QO
+//                   tiles of I_h(j) (analytic scheduler, ascending).  Per step five tcgen05 MMAs:
+//                     S^T  = K Q^T            (TMEM, 128 kv x 64 q)
+//                     dP^T = V dO^T           (TMEM)
+//                     dV  += P^T dO           (P^T as the TMEM operand)
+//                     dK  += dS^T Q           (dS^T as the TMEM operand)
+//                     dQ^T = K^T dS^T         (dS^T from shared memory; 128 d x 64 q in TMEM)
+//                   dK and dV stay in TMEM for the whole loop, all G heads included, so they need no
+//                   atomics (Algorithm 2 line 17 needs them only because it gives each QO head its
+//                   own program).  dQ^T is drained by a second warpgroup and added to the fp32
+//                   accumulator with red.global.add (Algorithm 2 line 15).
+//                   Warp roles: TMA producer / MMA issuer / compute warpgroup (P, dS) / dQ drain
+//                   warpgroup, connected by mbarriers; S^T is double buffered so that the MMAs of
+//                   steps n+1, n+2 overlap the element-wise work of step n.
+//   3. convert      dQ accumulator (already scaled) -> bf16.
+#include <cuda_bf16.h>
+
 #include "cowa_common.h"
+#include "cowa_ptx.cuh"
+#include "cowa_tma.h"
+
+using namespace cowa_ptx;
+
+namespace {
+
+constexpr int BKV = 128;  // KV rows per block (MMA M)
+constexpr int BQS = 64;   // QO rows per step (MMA N of S^T / dP^T)
+constexpr int NST = 3;    // Q / dO stages
+
+struct BwdArgs {
+  const float* lse2;   // [B*Hq, Tpad]  LSE * log2(e)
+  const float* delta;  // [B*Hq, Tpad]
+  float* dq_acc;       // [B*Hq, Tpad, D] fp32
+  unsigned int* status;
+  int B, Nq, Nk, Hq, Hkv, G, Tpad;
+  float scale, scale_log2;
+  CowaHeadWindows wins;
+};
+
+template <int D>
+struct BwdSmem {
+  static constexpr int kKV = BKV * D * 2;      // K or V tile
+  static constexpr int kQS = BQS * D * 2;      // Q or dO step tile
+  static constexpr int kStage = 2 * kQS;       // Q + dO
+  static constexpr int kDS = BKV * BQS * 2;    // dS^T tile (bf16)
+  static constexpr int oK = 0, oV = kKV, oStage = 2 * kKV, oDS = oStage + NST * kStage;
+  static constexpr int oVec = oDS + 2 * kDS;   // per stage: 64 floats lse2, 64 floats delta
+  static constexpr int oBar = oVec + NST * 512;
+  static constexpr int kBytes = oBar + 256 + 1024;
+};
+
+__device__ __forceinline__ void bulk_load_1d(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+
+__device__ __forceinline__ uint32_t interval_bits32(long long a, long long b, long long base) {
+  long long lo = a - base, hi = b - base;
+  if (lo < 0) lo = 0;
+  if (hi > 31) hi = 31;
+  if (lo > hi) return 0u;
+  return (0xFFFFFFFFu >> (31 - (int)(hi - lo))) << (int)lo;
+}
+
+__device__ __forceinline__ void red_add_f32(float* p, float v) {
+  asm volatile("red.global.add.f32 [%0], %1;" ::"l"(p), "f"(v) : "memory");
+}
+
+// named barrier for one 128-thread warpgroup
+__device__ __forceinline__ void wg_sync(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
+
+template <int D>
+__global__ void __launch_bounds__(320, 1)
+cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmdO,
+                const __grid_constant__ CUtensorMap tmdK, const __grid_constant__ CUtensorMap tmdV,
+                const __grid_constant__ BwdArgs a) {
+  using SM = BwdSmem<D>;
+  constexpr int NSLAB = D / 64;
+  constexpr int SLAB_KV = BKV * 128;  // bytes of one 64-wide slab of a 128-row tile
+  constexpr int SLAB_QS = BQS * 128;  // ... of a 64-row tile
+  // TMEM columns
+  constexpr uint32_t cS0 = 0, cDP = 128, cDQ = 192, cDK = 256, cDV = 384, TMEM_COLS = 512;
+  constexpr uint32_t ID_ST = idesc_bf16(128, BQS, 0, 0);   // S^T, dP^T
+  constexpr uint32_t ID_ACC = idesc_bf16(128, D, 0, 1);    // dV, dK (B = dO / Q, MN-major)
+  constexpr uint32_t ID_DQ = idesc_bf16(128, BQS, 1, 1);   // dQ^T (A = K^T, B = dS^T, both MN-major)
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sK = smem + SM::oK;
+  uint8_t* sV = smem + SM::oV;
+  uint8_t* sStage = smem + SM::oStage;
+  uint8_t* sDS = smem + SM::oDS;
+  float* sVec = reinterpret_cast<float*>(smem + SM::oVec);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::oBar);
+  uint64_t* bar_kv = bars + 0;
+  uint64_t* bar_ld_full = bars + 1;             // [NST]
+  uint64_t* bar_ld_empty = bars + 1 + NST;      // [NST]
+  uint64_t* bar_s_full = bars + 1 + 2 * NST;    // [2]
+  uint64_t* bar_dp_full = bars + 3 + 2 * NST;
+  uint64_t* bar_pds_ready = bars + 4 + 2 * NST; // count 128
+  uint64_t* bar_dq_full = bars + 5 + 2 * NST;
+  uint64_t* bar_dq_free = bars + 6 + 2 * NST;   // count 128
+  uint64_t* bar_done = bars + 7 + 2 * NST;
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 8 + 2 * NST);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  // ---- work item: KV tiles ascending (early tiles carry the most work) ----
+  int idx = blockIdx.x;
+  const int hk = idx % a.Hkv; idx /= a.Hkv;
+  const int b = idx % a.B; idx /= a.B;
+  const int j = idx;
+  const int off = a.Nk - a.Nq;
+  const int k0 = j * BKV, k1 = min(k0 + BKV, a.Nk) - 1;
+  const CowaWin w = a.wins.w[hk];
+  CowaRange rg[2];
+  cowa_bwd_ranges(w, k0, k1, off, a.Nq, BQS, rg);
+  const int cnt = cowa_range_len(rg[0]) + cowa_range_len(rg[1]);  // QO steps per head
+  const int N = cnt * a.G;
+  const int bhk = b * a.Hkv + hk;
+
+  if (tid == 0) {
+    mbar_init(bar_kv, 1);
+    for (int s = 0; s < NST; ++s) { mbar_init(bar_ld_full + s, 1); mbar_init(bar_ld_empty + s, 1); }
+    mbar_init(bar_s_full, 1); mbar_init(bar_s_full + 1, 1);
+    mbar_init(bar_dp_full, 1); mbar_init(bar_pds_ready, 128);
+    mbar_init(bar_dq_full, 1); mbar_init(bar_dq_free, 128); mbar_init(bar_done, 1);
+    fence_mbar_init();
+  }
+  if (warp == 0) {
+    __syncwarp();
+    tmem_alloc(tmem_holder, TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+
+  bool ok = true;
+
+  if (N > 0) {
+    if (warp == 0) {
+      // ================= TMA producer =================
+      if (lane == 0) {
+        prefetch_tmap(&tmQ); prefetch_tmap(&tmdO); prefetch_tmap(&tmK); prefetch_tmap(&tmV);
+        mbar_expect_tx(bar_kv, 2 * SM::kKV);
+        for (int s = 0; s < NSLAB; ++s) {
+          tma_load_3d(sK + s * SLAB_KV, &tmK, bar_kv, s * 64, k0, bhk);
+          tma_load_3d(sV + s * SLAB_KV, &tmV, bar_kv, s * 64, k0, bhk);
+        }
+        for (int n = 0; n < N && ok; ++n) {
+          const int st = n % NST;
+          if (n >= NST) ok = mbar_wait(bar_ld_empty + st, ((n / NST) - 1) & 1, a.status);
+          if (!ok) break;
+          const int g = n / cnt, i = cowa_bwd_tile_at(rg, n % cnt);
+          const int bhq = b * a.Hq + hk * a.G + g, q0 = i * BQS;
+          uint8_t* sQ = sStage + st * SM::kStage;
+          uint8_t* sdO = sQ + SM::kQS;
+          mbar_expect_tx(bar_ld_full + st, SM::kStage + 512);
+          for (int s = 0; s < NSLAB; ++s) {
+            tma_load_3d(sQ + s * SLAB_QS, &tmQ, bar_ld_full + st, s * 64, q0, bhq);
+            tma_load_3d(sdO + s * SLAB_QS, &tmdO, bar_ld_full + st, s * 64, q0, bhq);
+          }
+          bulk_load_1d(sVec + st * 128, a.lse2 + (size_t)bhq * a.Tpad + q0, 256, bar_ld_full + st);
+          bulk_load_1d(sVec + st * 128 + 64, a.delta + (size_t)bhq * a.Tpad + q0, 256, bar_ld_full + st);
+        }
+      }
+    } else if (warp == 1) {
+      // ================= MMA issuer =================
+      if (lane == 0) {
+        auto gemm_st = [&](uint32_t d_col, const uint8_t* sA, const uint8_t* sB) {  // [128 x 64] = A[128xD] B[64xD]^T
+#pragma unroll
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint32_t oa = (kk / 4) * SLAB_KV + (kk % 4) * 32, ob = (kk / 4) * SLAB_QS + (kk % 4) * 32;
+            mma_ss(tmem_base + d_col, smem_desc_sw128(smem_u32(sA) + oa, 16, 1024),
+                   smem_desc_sw128(smem_u32(sB) + ob, 16, 1024), ID_ST, kk > 0);
+          }
+        };
+        auto gemm_acc = [&](uint32_t d_col, uint32_t a_col, const uint8_t* sB, bool first) {  // [128 x D] += A^T-in-TMEM B
+#pragma unroll
+          for (int kk = 0; kk < BQS / 16; ++kk)
+            mma_ts(tmem_base + d_col, tmem_base + a_col + kk * 8,
+                   smem_desc_sw128(smem_u32(sB) + kk * 2048, SLAB_QS, 1024), ID_ACC, (!first || kk > 0) ? 1u : 0u);
+        };
+        auto gemm_dq = [&](const uint8_t* sB) {  // dQ^T[D x 64] = K^T dS^T
+#pragma unroll
+          for (int kk = 0; kk < BKV / 16; ++kk)
+            mma_ss(tmem_base + cDQ, smem_desc_sw128(smem_u32(sK) + kk * 2048, D == 128 ? SLAB_KV : 0, 1024),
+                   smem_desc_sw128(smem_u32(sB) + kk * 2048, 0, 1024), ID_DQ, kk > 0);
+        };
+        ok = mbar_wait(bar_kv, 0, a.status);
+        // prologue: S^T(0), dP^T(0), S^T(1)
+        ok = ok && mbar_wait(bar_ld_full + 0, 0, a.status);
+        if (ok) {
+          tc_fence_after();
+          gemm_st(cS0, sK, sStage);
+          mma_commit(bar_s_full + 0);
+          gemm_st(cDP, sV, sStage + SM::kQS);
+          mma_commit(bar_dp_full);
+        }
+        if (ok && N > 1) {
+          ok = mbar_wait(bar_ld_full + 1, 0, a.status);
+          if (ok) {
+            tc_fence_after();
+            gemm_st(cS0 + 64, sK, sStage + SM::kStage);
+            mma_commit(bar_s_full + 1);
+          }
+        }
+        for (int n = 0; n < N && ok; ++n) {
+          const int st = n % NST;
+          uint8_t* sQ = sStage + st * SM::kStage;
+          uint8_t* sdO = sQ + SM::kQS;
+          ok = mbar_wait(bar_pds_ready, n & 1, a.status);
+          if (!ok) break;
+          tc_fence_after();
+          gemm_acc(cDV, cS0 + (n & 1) * 64, sdO, n == 0);  // dV += P^T dO
+          gemm_acc(cDK, cDP, sQ, n == 0);                  // dK += dS^T Q
+          mma_commit(bar_ld_empty + st);
+          if (n + 1 < N) {                                 // dP^T(n+1): its stage was awaited one step ago
+            const int s1 = (n + 1) % NST;
+            gemm_st(cDP, sV, sStage + s1 * SM::kStage + SM::kQS);
+            mma_commit(bar_dp_full);
+          }
+          if (n + 2 < N) {                                 // S^T(n+2) into the buffer P^T(n) just left
+            const int s2 = (n + 2) % NST;
+            ok = mbar_wait(bar_ld_full + s2, ((n + 2) / NST) & 1, a.status);
+            if (!ok) break;
+            tc_fence_after();
+            gemm_st(cS0 + (n & 1) * 64, sK, sStage + s2 * SM::kStage);
+            mma_commit(bar_s_full + (n & 1));
+          }
+          if (n > 0) {
+            ok = mbar_wait(bar_dq_free, (n - 1) & 1, a.status);
+            if (!ok) break;
+            tc_fence_after();
+          }
+          gemm_dq(sDS + (n & 1) * SM::kDS);
+          mma_commit(bar_dq_full);
+        }
+        mma_commit(bar_done);
+      }
+    } else if (warp < 6) {
+      // ================= compute warpgroup: P^T and dS^T, one KV row per thread =================
+      const int r = (warp & 3) * 32 + lane;  // KV row = TMEM lane
+      const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+      const int kcol = k0 + r;               // key index of this thread
+      const long long kpos = (long long)kcol - off;  // first causal query of this key
+      for (int n = 0; n < N && ok; ++n) {
+        const int st = n % NST;
+        const int i = cowa_bwd_tile_at(rg, n % cnt);
+        const int q0 = i * BQS;
+        const bool full = cowa_tile_full(w, q0, BQS, k0, BKV, off, a.Nq, a.Nk);
+        uint32_t mk[2] = {0xFFFFFFFFu, 0xFFFFFFFFu};
+        if (!full) {
+          const long long qend = a.Nq - 1;
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {
+            const long long base = q0 + c * 32;
+            uint32_t m = interval_bits32(kpos, min(kpos + w.n - 1, qend), base);
+            if (w.l > 0)
+              m |= interval_bits32(kpos + w.n + w.g, min(kpos + (long long)w.n + w.g + w.l - 1, qend), base);
+            if (kcol < w.s) m |= interval_bits32(kpos, qend, base);
+            mk[c] = kcol < a.Nk ? m : 0u;
+          }
+        }
+        const float* lse2 = sVec + st * 128;
+        const float* dlt = lse2 + 64;
+        ok = mbar_wait(bar_ld_full + st, (n / NST) & 1, a.status);
+        ok = ok && mbar_wait(bar_s_full + (n & 1), (n >> 1) & 1, a.status);
+        if (!ok) break;
+        tc_fence_after();
+        float p[64];
+        uint32_t pk[32];
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t sr[32];
+          tmem_ld32(t_lane + cS0 + (n & 1) * 64 + c * 32, sr);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            float x = ex2(fmaf(__uint_as_float(sr[e]), a.scale_log2, -lse2[c * 32 + e]));
+            if (!full) x = (mk[c] >> e) & 1u ? x : 0.f;
+            p[c * 32 + e] = x;
+          }
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) pk[c * 16 + e / 2] = pack_bf16(p[c * 32 + e], p[c * 32 + e + 1]);
+        }
+        tmem_st32(t_lane + cS0 + (n & 1) * 64, pk);  // P^T over the first 32 columns of this S^T buffer
+
+        ok = mbar_wait(bar_dp_full, n & 1, a.status);
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t dk_[32];
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t dr[32];
+          tmem_ld32(t_lane + cDP + c * 32, dr);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            const float d0 = p[c * 32 + e] * (__uint_as_float(dr[e]) - dlt[c * 32 + e]);
+            const float d1 = p[c * 32 + e + 1] * (__uint_as_float(dr[e + 1]) - dlt[c * 32 + e + 1]);
+            dk_[c * 16 + e / 2] = pack_bf16(d0, d1);
+          }
+        }
+        tmem_st32(t_lane + cDP, dk_);  // dS^T over the first 32 columns of dP^T
+        // dS^T also to shared memory (row r = 128 B = 8 chunks, 128B swizzle) for the dQ^T product
+        uint8_t* ds_row = sDS + (n & 1) * SM::kDS + r * 128;
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch)
+          *reinterpret_cast<uint4*>(ds_row + ((ch ^ (r & 7)) << 4)) =
+              make_uint4(dk_[ch * 4], dk_[ch * 4 + 1], dk_[ch * 4 + 2], dk_[ch * 4 + 3]);
+        tmem_wait_st();
+        tc_fence_before();
+        fence_proxy_async_smem();
+        mbar_arrive(bar_pds_ready);
+      }
+    } else {
+      // ================= dQ drain warpgroup: one d column of dQ^T per thread =================
+      const int d = (warp & 3) * 32 + lane;
+      const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+      for (int n = 0; n < N && ok; ++n) {
+        const int g = n / cnt, i = cowa_bwd_tile_at(rg, n % cnt);
+        const int bhq = b * a.Hq + hk * a.G + g, q0 = i * BQS;
+        ok = mbar_wait(bar_dq_full, n & 1, a.status);
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t v0[32], v1[32];
+        tmem_ld32(t_lane + cDQ, v0);
+        tmem_ld32(t_lane + cDQ + 32, v1);
+        tmem_wait_ld();
+        tc_fence_before();
+        mbar_arrive(bar_dq_free);
+        if (d < D) {
+          float* dst = a.dq_acc + ((size_t)bhq * a.Tpad + q0) * D + d;
+          const int nrow = min(BQS, a.Nq - q0);
+#pragma unroll
+          for (int c = 0; c < 32; ++c)
+            if (c < nrow) red_add_f32(dst + (size_t)c * D, __uint_as_float(v0[c]) * a.scale);
+#pragma unroll
+          for (int c = 0; c < 32; ++c)
+            if (c + 32 < nrow) red_add_f32(dst + (size_t)(c + 32) * D, __uint_as_float(v1[c]) * a.scale);
+        }
+      }
+    }
+  }
+
+  // ---- epilogue: dK (compute warpgroup) and dV (drain warpgroup) -> bf16 -> shared -> TMA store ----
+  if (warp >= 2) {
+    const bool is_dk = warp < 6;
+    const int r = (warp & 3) * 32 + lane;
+    const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+    if (N > 0) ok = mbar_wait(bar_done, 0, a.status) && ok;
+    tc_fence_after();
+    uint8_t* sOut = sStage + (is_dk ? 0 : SM::kKV);
+    const float mul = is_dk ? a.scale : 1.f;
+#pragma unroll
+    for (int c = 0; c < D / 32; ++c) {
+      uint32_t ov[32];
+      if (N > 0 && ok) {
+        tmem_ld32(t_lane + (is_dk ? cDK : cDV) + c * 32, ov);
+        tmem_wait_ld();
+      } else {
+#pragma unroll
+        for (int e = 0; e < 32; ++e) ov[e] = 0u;
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        uint4 v;
+        v.x = pack_bf16(__uint_as_float(ov[q * 8 + 0]) * mul, __uint_as_float(ov[q * 8 + 1]) * mul);
+        v.y = pack_bf16(__uint_as_float(ov[q * 8 + 2]) * mul, __uint_as_float(ov[q * 8 + 3]) * mul);
+        v.z = pack_bf16(__uint_as_float(ov[q * 8 + 4]) * mul, __uint_as_float(ov[q * 8 + 5]) * mul);
+        v.w = pack_bf16(__uint_as_float(ov[q * 8 + 6]) * mul, __uint_as_float(ov[q * 8 + 7]) * mul);
+        const int d0 = c * 32 + q * 8;
+        const int slab = d0 / 64, chunk = (d0 % 64) / 8;
+        *reinterpret_cast<uint4*>(sOut + slab * SLAB_KV + r * 128 + ((chunk ^ (r & 7)) << 4)) = v;
+      }
+    }
+    fence_proxy_async_smem();
+    wg_sync(is_dk ? 1 : 2);
+    if (r == 0 && ok) {
+      for (int s = 0; s < NSLAB; ++s) tma_store_3d(is_dk ? &tmdK : &tmdV, sOut + s * SLAB_KV, s * 64, k0, bhk);
+      tma_commit_group();
+      tma_wait_group<0>();
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    __syncwarp();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+// Delta = rowsum(O * dO), lse2 = LSE * log2(e); rows in [T, Tpad) get lse2 = +inf, Delta = 0.
+template <int D>
+__global__ void cowa_bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ d_o,
+                                           const float* __restrict__ lse, float* __restrict__ lse2,
+                                           float* __restrict__ delta, int T, int Tpad, long long BH) {
+  constexpr int TPR = D / 8;  // threads per row (16 bytes each)
+  const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long row = gid / TPR;
+  const int part = (int)(gid % TPR);
+  if (row >= BH * Tpad) return;
+  const long long bh = row / Tpad;
+  const int t = (int)(row % Tpad);
+  float s = 0.f;
+  if (t < T) {
+    const size_t base = ((size_t)bh * T + t) * D + part * 8;
+    const uint4 x = *reinterpret_cast<const uint4*>(o + base);
+    const uint4 y = *reinterpret_cast<const uint4*>(d_o + base);
+    const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      s = fmaf(__uint_as_float(xs[i] << 16), __uint_as_float(ys[i] << 16), s);
+      s = fmaf(__uint_as_float(xs[i] & 0xffff0000u), __uint_as_float(ys[i] & 0xffff0000u), s);
+    }
+  }
+#pragma unroll
+  for (int o_ = TPR / 2; o_ > 0; o_ >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o_);
+  if (part == 0) {
+    delta[row] = s;
+    lse2[row] = t < T ? lse[(size_t)bh * T + t] * 1.4426950408889634f : INFINITY;
+  }
+}
+
+template <int D>
+__global__ void cowa_bwd_convert_dq_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dq, int T,
+                                           int Tpad, long long BH) {
+  const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;  // one thread per 8 elements
+  const long long total = BH * T * (D / 8);
+  if (gid >= total) return;
+  const long long row = gid / (D / 8);
+  const int part = (int)(gid % (D / 8));
+  const long long bh = row / T;
+  const int t = (int)(row % T);
+  const float4* src = reinterpret_cast<const float4*>(acc + ((size_t)bh * Tpad + t) * D + part * 8);
+  const float4 x = src[0], y = src[1];
+  uint4 v;
+  v.x = pack_bf16(x.x, x.y); v.y = pack_bf16(x.z, x.w); v.z = pack_bf16(y.x, y.y); v.w = pack_bf16(y.z, y.w);
+  *reinterpret_cast<uint4*>(dq + ((size_t)bh * T + t) * D + part * 8) = v;
+}
+
+size_t ws_bytes(int B, int T, int Hq, int D) {
+  const size_t Tpad = ((size_t)T + BQS - 1) / BQS * BQS;
+  return (size_t)B * Hq * Tpad * ((size_t)D + 2) * sizeof(float);
+}
+
+template <int D>
+int launch_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* d_o,
+               void* dq, void* dk, void* dv, int B, int T, int Hq, int Hkv, const cowa_params_t* p,
+               const CowaHeadWindows& hw, void* ws, cudaStream_t st) {
+  const int Tpad = (T + BQS - 1) / BQS * BQS;
+  const long long BH = (long long)B * Hq;
+  float* dq_acc = static_cast<float*>(ws);
+  float* lse2 = dq_acc + (size_t)BH * Tpad * D;
+  float* delta = lse2 + (size_t)BH * Tpad;
+  COWA_CUDA_TRY(cudaMemsetAsync(dq_acc, 0, (size_t)BH * Tpad * D * sizeof(float), st));
+  {
+    const long long threads = BH * Tpad * (D / 8);
+    cowa_bwd_preprocess_kernel<D><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(
+        static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse, lse2, delta, T, Tpad, BH);
+    COWA_CUDA_TRY(cudaGetLastError());
+  }
+  CUtensorMap mq, mk, mv, mdo, mdk, mdv;
+  int rc;
+  if ((rc = cowa::make_tensor_map_3d(&mq, q, cowa::MapType::BF16, D, T, BH, 64, BQS))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mdo, d_o, cowa::MapType::BF16, D, T, BH, 64, BQS))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mk, k, cowa::MapType::BF16, D, T, (long long)B * Hkv, 64, BKV))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mv, v, cowa::MapType::BF16, D, T, (long long)B * Hkv, 64, BKV))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mdk, dk, cowa::MapType::BF16, D, T, (long long)B * Hkv, 64, BKV))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mdv, dv, cowa::MapType::BF16, D, T, (long long)B * Hkv, 64, BKV))) return rc;
+  BwdArgs a;
+  a.lse2 = lse2; a.delta = delta; a.dq_acc = dq_acc;
+  a.status = cowa::device_status_word();
+  if (!a.status) return COWA_ERR_CUDA;
+  a.B = B; a.Nq = T; a.Nk = T; a.Hq = Hq; a.Hkv = Hkv; a.G = Hq / Hkv; a.Tpad = Tpad;
+  a.scale = p->softmax_scale;
+  a.scale_log2 = p->softmax_scale * 1.4426950408889634f;
+  a.wins = hw;
+  COWA_CUDA_TRY(cudaFuncSetAttribute(cowa_bwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     BwdSmem<D>::kBytes));
+  const long long nblocks = (long long)((T + BKV - 1) / BKV) * B * Hkv;
+  if (nblocks > 0x7FFFFFFFll) return COWA_ERR_UNSUPPORTED;
+  cowa_bwd_kernel<D><<<(unsigned)nblocks, 320, BwdSmem<D>::kBytes, st>>>(mq, mk, mv, mdo, mdk, mdv, a);
+  COWA_CUDA_TRY(cudaGetLastError());
+  {
+    const long long threads = BH * T * (D / 8);
+    cowa_bwd_convert_dq_kernel<D><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(
+        dq_acc, static_cast<__nv_bfloat16*>(dq), T, Tpad, BH);
+    COWA_CUDA_TRY(cudaGetLastError());
+  }
+  return COWA_OK;
+}
+
+}  // namespace
 
 extern "C" {
 
 size_t cowa_bwd_workspace_bytes(int B, int T, int Hq, int Hkv, int D, const cowa_params_t* p) {
-  (void)Hkv; (void)D; (void)p;
-  if (B <= 0 || T <= 0 || Hq <= 0) return 0;
-  return (size_t)B * Hq * T * sizeof(float);
+  (void)Hkv; (void)p;
+  if (B <= 0 || T <= 0 || Hq <= 0 || D <= 0) return 0;
+  return ws_bytes(B, T, Hq, D);
 }
 
 int cowa_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* d_o,
              void* dq, void* dk, void* dv, int B, int T, int Hq, int Hkv, int D, const cowa_params_t* p,
              void* workspace, size_t workspace_bytes, void* stream) {
-  (void)T; (void)B; (void)Hq; (void)Hkv; (void)D; (void)workspace_bytes; (void)stream;
   if (!q || !k || !v || !o || !lse || !d_o || !dq || !dk || !dv || !p || !workspace) return COWA_ERR_INVALID_ARG;
-  return COWA_ERR_UNSUPPORTED;
+  if (B <= 0 || T <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0) return COWA_ERR_INVALID_ARG;
+  if (!(p->softmax_scale > 0.f)) return COWA_ERR_INVALID_ARG;
+  if (D != 64 && D != 128) return COWA_ERR_UNSUPPORTED;
+  const void* ptrs[] = {q, k, v, o, d_o, dq, dk, dv, workspace};
+  for (const void* x : ptrs)
+    if (!cowa::aligned16(x)) return COWA_ERR_MISALIGNED;
+  if (workspace_bytes < ws_bytes(B, T, Hq, D)) return COWA_ERR_WORKSPACE_TOO_SMALL;
+  CowaHeadWindows hw;
+  int rc = cowa::resolve_windows(T, Hkv, p, &hw);
+  if (rc != COWA_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  return D == 128 ? launch_bwd<128>(q, k, v, o, lse, d_o, dq, dk, dv, B, T, Hq, Hkv, p, hw, workspace, st)
+                  : launch_bwd<64>(q, k, v, o, lse, d_o, dq, dk, dv, B, T, Hq, Hkv, p, hw, workspace, st);
 }
 
 }  // extern "C"

@@ -1,6 +1,9 @@
 """GPU parity: the CUDA path (through the C ABI) against the float64 CPU oracle on the same
-seeded bf16 inputs.  Tolerances (bf16 inputs/outputs, fp32 accumulation, P rounded to bf16
-before its second product): O and gradients max-abs 2e-2 and mean-abs 2e-3, LSE max-abs 1e-3."""
+seeded bf16 inputs.  Tolerances (bf16 inputs/outputs, fp32 accumulation, P and dS rounded to bf16
+before their second product): O and gradients max-abs 2e-2 and mean-abs 2e-3, LSE max-abs 1e-3.
+Gradients are stored as bf16 and reach magnitudes above 4, where rounding the exact value to bf16
+alone costs up to |x| * 2^-8 (half an ulp); the gradient check therefore allows
+2e-2 + 2^-8 * |reference| per element.  The mean-abs bound is unchanged."""
 import numpy as np
 import pytest
 import torch
@@ -15,12 +18,20 @@ TOL_MAX, TOL_MEAN, TOL_LSE = 2e-2, 2e-3, 1e-3
 DEV = "cuda"
 
 
-def check(name, got, want, tol_max=TOL_MAX, tol_mean=TOL_MEAN):
+def check(name, got, want, tol_max=TOL_MAX, tol_mean=TOL_MEAN, rtol=0.0):
     got = np.asarray(got, dtype=np.float64)
     err = np.abs(got - want)
     assert np.isfinite(got).all(), f"{name}: non-finite output"
-    assert err.max() <= tol_max, f"{name}: max-abs {err.max():.3e} > {tol_max}"
+    excess = err - rtol * np.abs(want)
+    assert excess.max() <= tol_max, f"{name}: max-abs {err.max():.3e} (excess {excess.max():.3e}) > {tol_max}"
     assert err.mean() <= tol_mean, f"{name}: mean-abs {err.mean():.3e} > {tol_mean}"
+
+
+BF16_HALF_ULP = 2.0 ** -8
+
+
+def check_grad(name, got, want):
+    check(name, got, want, rtol=BF16_HALF_ULP)
 
 
 def run_fwd(q, k, v, params):
@@ -101,6 +112,94 @@ def test_fwd_8k_config_sampled_heads():
                                       wd, scale, 13, rows)
     check("dup lse", lse[0, 13].cpu().numpy(), lse_ref, TOL_LSE, TOL_LSE)
     check("dup o", o[0, 13].float().cpu().numpy(), o_ref)
+
+
+# ------------------------------------------------------------------ backward
+
+def run_fwd_bwd(q, k, v, d_o, params):
+    B, Hq, T, D = q.shape
+    Hkv = k.shape[1]
+    o, lse = run_fwd(q, k, v, params)
+    dq, dk, dv = (torch.full_like(x, float("nan")) for x in (q, k, v))
+    nbytes = cowa.cowa_bwd_workspace_bytes(B, T, Hq, Hkv, D, params)
+    ws = torch.empty(nbytes + 64, dtype=torch.uint8, device=q.device)
+    ws.fill_(0xFF)  # the workspace needs no initialisation by the caller
+    cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, params, ws[:nbytes])
+    torch.cuda.synchronize()
+    cowa.cowa_check_device_status()
+    assert (ws[nbytes:] == 0xFF).all(), "backward wrote past its workspace"
+    return dq, dk, dv
+
+
+def bwd_case(B, T, Hq, Hkv, D, sink, local, seed=51, windows=None, full_attn=False):
+    q, k, v, d_o = cowa_inputs.make_train_inputs(seed, B, T, Hq, Hkv, D)
+    scale = cowa_inputs.softmax_scale(D)
+    params = cowa.make_params(sink=sink, local=local, softmax_scale=scale, windows=windows, full_attn=full_attn)
+    dq, dk, dv = run_fwd_bwd(q.to(DEV), k.to(DEV), v.to(DEV), d_o.to(DEV), params)
+    if full_attn:
+        ws = [(0, T, 0, 0)] * Hkv
+    else:
+        ws = windows if windows is not None else orc.default_windows(T, Hkv, sink, local)
+    f = cowa_inputs.to_f64
+    for b in range(B):
+        dq_r, dk_r, dv_r = orc.backward(f(q[b]), f(k[b]), f(v[b]), f(d_o[b]), ws, scale)
+        check_grad(f"dq[b={b}]", dq[b].float().cpu().numpy(), dq_r)
+        check_grad(f"dk[b={b}]", dk[b].float().cpu().numpy(), dk_r)
+        check_grad(f"dv[b={b}]", dv[b].float().cpu().numpy(), dv_r)
+
+
+def test_bwd_tiny_config():
+    c = cowa_inputs.CONFIGS["tiny"]
+    bwd_case(c["B"], c["T"], c["Hq"], c["Hkv"], c["D"], c["sink"], c["local"], seed=c["index"])
+
+
+@pytest.mark.parametrize("B,T,Hq,Hkv,D,sink,local", [
+    (1, 64, 1, 1, 128, 0, 64),        # a single step
+    (1, 256, 2, 1, 128, 0, 1),        # near = 1
+    (2, 640, 8, 2, 128, 16, 100),     # bands not tile aligned, G = 4
+    (1, 1000, 4, 4, 64, 7, 33),       # ragged tail, G = 1, D = 64
+    (1, 1100, 8, 1, 128, 5, 9),       # H_k = 1, G = 8
+    (1, 512, 4, 2, 128, 300, 300),    # dense causal
+    (1, 1536, 16, 2, 64, 200, 64),    # wide sink
+    (1, 77, 2, 2, 128, 3, 4),         # shorter than one tile
+])
+def test_bwd_shapes(B, T, Hq, Hkv, D, sink, local):
+    bwd_case(B, T, Hq, Hkv, D, sink, local)
+
+
+def test_bwd_full_attn_and_explicit_windows():
+    bwd_case(1, 900, 4, 2, 128, 0, 1, full_attn=True)
+    bwd_case(1, 1024, 4, 2, 64, 64, 128, windows=orc.duplicated_windows(1024, 2, 64, 128, 1))
+    bwd_case(1, 700, 2, 2, 128, 0, 1, windows=[(0, 50, 100, 200), (20, 10, 0, 0)])
+
+
+def test_bwd_dkdv_bitwise_repeatable():
+    # dK and dV are accumulated in a fixed order inside one block: two runs must agree bit for bit.
+    q, k, v, d_o = cowa_inputs.make_train_inputs(52, 1, 2048, 8, 2, 128, device=DEV)
+    params = cowa.make_params(sink=32, local=256, softmax_scale=cowa_inputs.softmax_scale(128))
+    _, dk1, dv1 = run_fwd_bwd(q, k, v, d_o, params)
+    _, dk2, dv2 = run_fwd_bwd(q, k, v, d_o, params)
+    assert torch.equal(dk1, dk2) and torch.equal(dv1, dv2)
+
+
+def test_bwd_8k_config_sampled():
+    c = cowa_inputs.CONFIGS["8k"]
+    B, T, Hq, Hkv, D = c["B"], c["T"], c["Hq"], c["Hkv"], c["D"]
+    q, k, v, d_o = cowa_inputs.make_train_inputs(c["index"], B, T, Hq, Hkv, D)
+    scale = cowa_inputs.softmax_scale(D)
+    params = cowa.make_params(sink=c["sink"], local=c["local"], softmax_scale=scale)
+    dq, dk, dv = run_fwd_bwd(q.to(DEV), k.to(DEV), v.to(DEV), d_o.to(DEV), params)
+    ws = orc.default_windows(T, Hkv, c["sink"], c["local"])
+    f = cowa_inputs.to_f64
+    # dQ: whole heads; dK/dV: KV tiles incl. the sink tile, a band edge and the last tile
+    for b, h in [(0, 1), (1, 14)]:
+        ref = orc.backward_dq_rows(f(q[b]), f(k[b]), f(v[b]), f(d_o[b]), ws, scale, h, np.arange(T))
+        check_grad(f"dq[{b},{h}]", dq[b, h].float().cpu().numpy(), ref)
+    for b, hk, tile in [(0, 0, 0), (0, 2, 17), (1, 3, 63), (1, 1, 30)]:
+        cols = np.arange(tile * 128, tile * 128 + 128)
+        dk_r, dv_r = orc.backward_dkdv_cols(f(q[b]), f(k[b]), f(v[b]), f(d_o[b]), ws, scale, hk, cols)
+        check_grad(f"dk[{b},{hk},{tile}]", dk[b, hk, cols].float().cpu().numpy(), dk_r)
+        check_grad(f"dv[{b},{hk},{tile}]", dv[b, hk, cols].float().cpu().numpy(), dv_r)
 
 
 # ------------------------------------------------------------------ decode
