@@ -209,8 +209,10 @@ def run_cuda(args):
     dev = torch.device("cuda", torch.cuda.current_device())
     peaks, peak_src = load_peaks()
 
-    ct = cowa_inputs.CONFIGS[TRAIN_CFG]
-    cd = cowa_inputs.CONFIGS[DECODE_CFG]
+    ct = cowa_inputs.CONFIGS[args.train_cfg]
+    cd = dict(cowa_inputs.CONFIGS[DECODE_CFG])
+    if args.decode_batch:
+        cd["B"] = args.decode_batch
     B, T, Hq, Hkv, D = ct["B"], ct["T"], ct["Hq"], ct["Hkv"], ct["D"]
     scale = cowa_inputs.softmax_scale(D)
     p_train = cowa.make_params(sink=ct["sink"], local=ct["local"], softmax_scale=scale)
@@ -382,10 +384,10 @@ def run_cuda(args):
                          f"configuration, {t:.1f} s; legal-pair FLOPs"}
 
     line = {
-        "metric": "cowa_train_tflops_visited_tiles_128k", "value": value, "unit": "TFLOP/s", "n_gpus": world,
+        "metric": "cowa_train_tflops_visited_tiles_" + args.train_cfg, "value": value, "unit": "TFLOP/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": TRAIN_CFG, "decode_workload": DECODE_CFG, "B": B, "T": T, "Hq": Hq, "Hkv": Hkv,
+        "config": {"workload": args.train_cfg, "decode_workload": DECODE_CFG, "decode_batch": cd["B"], "B": B, "T": T, "Hq": Hq, "Hkv": Hkv,
                    "D": D, "sink": ct["sink"], "near": ct["local"],
                    "phases": ["fwd"] + (["bwd"] if have_bwd else []) + ["decode"],
                    "l2": "inputs larger than L2 (2.6 GB training tensors, 0.57 GB visible KV cache)",
@@ -413,6 +415,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--train-cfg", default=TRAIN_CFG, choices=["8k", "32k", "128k"],
+                    help="training configuration (default: the 128K headline; smaller ones are for profiling)")
+    ap.add_argument("--decode-batch", type=int, default=0, help="override the decode batch (profiling)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

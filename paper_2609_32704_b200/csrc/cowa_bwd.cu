@@ -14,13 +14,18 @@
 //                     dQ^T = K^T dS^T         (dS^T from shared memory; 128 d x 64 q in TMEM)
 //                   dK and dV stay in TMEM for the whole loop, all G heads included, so they need no
 //                   atomics (Algorithm 2 line 17 needs them only because it gives each QO head its
-//                   own program).  dQ^T is drained by a second warpgroup and added to the fp32
-//                   accumulator with red.global.add (Algorithm 2 line 15).
-//                   Warp roles: TMA producer / MMA issuer / compute warpgroup (P, dS) / dQ drain
-//                   warpgroup, connected by mbarriers; S^T is double buffered so that the MMAs of
-//                   steps n+1, n+2 overlap the element-wise work of step n.
+//                   own program).  dQ^T is drained by a separate warpgroup through shared memory and
+//                   added to the fp32 accumulator with TMA bulk reductions (Algorithm 2 line 15).
+//                   Warp roles: TMA producer / MMA issuer / two compute warpgroups (P, dS; 32 query
+//                   columns each) / dQ drain warpgroup, connected by mbarriers; S^T is double
+//                   buffered so that the MMAs of steps n+1, n+2 overlap the element-wise work of
+//                   step n.  Blocks are ordered sink tiles first (they meet every query tile), then
+//                   head by head with ascending KV tile, so that the blocks in flight sweep the same
+//                   dQ rows at nearly the same time and the reductions hit in L2.
 //   3. convert      dQ accumulator (already scaled) -> bf16.
 #include <cuda_bf16.h>
+
+#include <algorithm>
 
 #include "cowa_common.h"
 #include "cowa_ptx.cuh"
@@ -40,6 +45,7 @@ struct BwdArgs {
   float* dq_acc;       // [B*Hq, Tpad, D] fp32
   unsigned int* status;
   int B, Nq, Nk, Hq, Hkv, G, Tpad;
+  int sink_tiles;      // KV tiles per head that hold sink columns (launched first)
   float scale, scale_log2;
   CowaHeadWindows wins;
 };
@@ -52,7 +58,9 @@ struct BwdSmem {
   static constexpr int kDS = BKV * BQS * 2;    // dS^T tile (bf16)
   static constexpr int oK = 0, oV = kKV, oStage = 2 * kKV, oDS = oStage + NST * kStage;
   static constexpr int oVec = oDS + 2 * kDS;   // per stage: 64 floats lse2, 64 floats delta
-  static constexpr int oBar = oVec + NST * 512;
+  static constexpr int oDQ = oVec + NST * 512;  // dQ staging: 32 query rows x D fp32
+  static constexpr int kDQ = 32 * D * 4;
+  static constexpr int oBar = oDQ + kDQ;
   static constexpr int kBytes = oBar + 256 + 1024;
 };
 
@@ -71,19 +79,15 @@ __device__ __forceinline__ uint32_t interval_bits32(long long a, long long b, lo
   return (0xFFFFFFFFu >> (31 - (int)(hi - lo))) << (int)lo;
 }
 
-__device__ __forceinline__ void red_add_f32(float* p, float v) {
-  asm volatile("red.global.add.f32 [%0], %1;" ::"l"(p), "f"(v) : "memory");
-}
-
 // named barrier for one 128-thread warpgroup
 __device__ __forceinline__ void wg_sync(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
 
 template <int D>
-__global__ void __launch_bounds__(320, 1)
+__global__ void __launch_bounds__(512, 1)
 cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmdO,
                 const __grid_constant__ CUtensorMap tmdK, const __grid_constant__ CUtensorMap tmdV,
-                const __grid_constant__ BwdArgs a) {
+                const __grid_constant__ CUtensorMap tmdQ, const __grid_constant__ BwdArgs a) {
   using SM = BwdSmem<D>;
   constexpr int NSLAB = D / 64;
   constexpr int SLAB_KV = BKV * 128;  // bytes of one 64-wide slab of a 128-row tile
@@ -101,13 +105,14 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   uint8_t* sStage = smem + SM::oStage;
   uint8_t* sDS = smem + SM::oDS;
   float* sVec = reinterpret_cast<float*>(smem + SM::oVec);
+  float* sDQ = reinterpret_cast<float*>(smem + SM::oDQ);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::oBar);
   uint64_t* bar_kv = bars + 0;
   uint64_t* bar_ld_full = bars + 1;             // [NST]
   uint64_t* bar_ld_empty = bars + 1 + NST;      // [NST]
   uint64_t* bar_s_full = bars + 1 + 2 * NST;    // [2]
   uint64_t* bar_dp_full = bars + 3 + 2 * NST;
-  uint64_t* bar_pds_ready = bars + 4 + 2 * NST; // count 128
+  uint64_t* bar_pds_ready = bars + 4 + 2 * NST; // count 256
   uint64_t* bar_dq_full = bars + 5 + 2 * NST;
   uint64_t* bar_dq_free = bars + 6 + 2 * NST;   // count 128
   uint64_t* bar_done = bars + 7 + 2 * NST;
@@ -115,11 +120,19 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-  // ---- work item: KV tiles ascending (early tiles carry the most work) ----
-  int idx = blockIdx.x;
-  const int hk = idx % a.Hkv; idx /= a.Hkv;
-  const int b = idx % a.B; idx /= a.B;
-  const int j = idx;
+  // ---- work item: sink tiles of every head first, then head-major with ascending KV tile ----
+  int hk, b, j;
+  {
+    int idx = blockIdx.x;
+    const int nKV = (a.Nk + BKV - 1) / BKV, nsk = a.sink_tiles, nhead = a.B * a.Hkv;
+    if (idx < nsk * nhead) {
+      j = idx / nhead; idx %= nhead;
+    } else {
+      idx -= nsk * nhead;
+      j = nsk + idx % (nKV - nsk); idx /= (nKV - nsk);
+    }
+    hk = idx % a.Hkv; b = idx / a.Hkv;
+  }
   const int off = a.Nk - a.Nq;
   const int k0 = j * BKV, k1 = min(k0 + BKV, a.Nk) - 1;
   const CowaWin w = a.wins.w[hk];
@@ -133,7 +146,7 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     mbar_init(bar_kv, 1);
     for (int s = 0; s < NST; ++s) { mbar_init(bar_ld_full + s, 1); mbar_init(bar_ld_empty + s, 1); }
     mbar_init(bar_s_full, 1); mbar_init(bar_s_full + 1, 1);
-    mbar_init(bar_dp_full, 1); mbar_init(bar_pds_ready, 128);
+    mbar_init(bar_dp_full, 1); mbar_init(bar_pds_ready, 256);
     mbar_init(bar_dq_full, 1); mbar_init(bar_dq_free, 128); mbar_init(bar_done, 1);
     fence_mbar_init();
   }
@@ -189,8 +202,8 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         };
         auto gemm_acc = [&](uint32_t d_col, uint32_t a_col, const uint8_t* sB, bool first) {  // [128 x D] += A^T-in-TMEM B
 #pragma unroll
-          for (int kk = 0; kk < BQS / 16; ++kk)
-            mma_ts(tmem_base + d_col, tmem_base + a_col + kk * 8,
+          for (int kk = 0; kk < BQS / 16; ++kk)  // A: query columns 0-31 at a_col, 32-63 at a_col + 32
+            mma_ts(tmem_base + d_col, tmem_base + a_col + (kk & 1) * 8 + (kk >> 1) * 32,
                    smem_desc_sw128(smem_u32(sB) + kk * 2048, SLAB_QS, 1024), ID_ACC, (!first || kk > 0) ? 1u : 0u);
         };
         auto gemm_dq = [&](const uint8_t* sB) {  // dQ^T[D x 64] = K^T dS^T
@@ -250,115 +263,124 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         }
         mma_commit(bar_done);
       }
-    } else if (warp < 6) {
-      // ================= compute warpgroup: P^T and dS^T, one KV row per thread =================
+    } else if (warp >= 4 && warp < 12) {
+      // ======== two compute warpgroups: P^T and dS^T, one KV row per thread, 32 query columns each ========
+      const int half = (warp - 4) >> 2;      // 0: query columns 0-31, 1: 32-63
       const int r = (warp & 3) * 32 + lane;  // KV row = TMEM lane
       const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
       const int kcol = k0 + r;               // key index of this thread
       const long long kpos = (long long)kcol - off;  // first causal query of this key
+      const float2 sc2 = make_float2(a.scale_log2, a.scale_log2);
       for (int n = 0; n < N && ok; ++n) {
         const int st = n % NST;
         const int i = cowa_bwd_tile_at(rg, n % cnt);
         const int q0 = i * BQS;
         const bool full = cowa_tile_full(w, q0, BQS, k0, BKV, off, a.Nq, a.Nk);
-        uint32_t mk[2] = {0xFFFFFFFFu, 0xFFFFFFFFu};
+        uint32_t mk = 0xFFFFFFFFu;
         if (!full) {
-          const long long qend = a.Nq - 1;
-#pragma unroll
-          for (int c = 0; c < 2; ++c) {
-            const long long base = q0 + c * 32;
-            uint32_t m = interval_bits32(kpos, min(kpos + w.n - 1, qend), base);
-            if (w.l > 0)
-              m |= interval_bits32(kpos + w.n + w.g, min(kpos + (long long)w.n + w.g + w.l - 1, qend), base);
-            if (kcol < w.s) m |= interval_bits32(kpos, qend, base);
-            mk[c] = kcol < a.Nk ? m : 0u;
-          }
+          const long long qend = a.Nq - 1, base = q0 + half * 32;
+          uint32_t m = interval_bits32(kpos, min(kpos + w.n - 1, qend), base);
+          if (w.l > 0)
+            m |= interval_bits32(kpos + w.n + w.g, min(kpos + (long long)w.n + w.g + w.l - 1, qend), base);
+          if (kcol < w.s) m |= interval_bits32(kpos, qend, base);
+          mk = kcol < a.Nk ? m : 0u;
         }
-        const float* lse2 = sVec + st * 128;
-        const float* dlt = lse2 + 64;
+        const float* lse2 = sVec + st * 128 + half * 32;
+        const float* dlt = sVec + st * 128 + 64 + half * 32;
+        const uint32_t sbuf = cS0 + (n & 1) * 64 + half * 32;  // this half's S^T columns; P^T goes over the first 16
         ok = mbar_wait(bar_ld_full + st, (n / NST) & 1, a.status);
         ok = ok && mbar_wait(bar_s_full + (n & 1), (n >> 1) & 1, a.status);
         if (!ok) break;
         tc_fence_after();
-        float p[64];
-        uint32_t pk[32];
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
+        float p[32];
+        {
           uint32_t sr[32];
-          tmem_ld32(t_lane + cS0 + (n & 1) * 64 + c * 32, sr);
-          tmem_wait_ld();
-#pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            float x = ex2(fmaf(__uint_as_float(sr[e]), a.scale_log2, -lse2[c * 32 + e]));
-            if (!full) x = (mk[c] >> e) & 1u ? x : 0.f;
-            p[c * 32 + e] = x;
-          }
-#pragma unroll
-          for (int e = 0; e < 32; e += 2) pk[c * 16 + e / 2] = pack_bf16(p[c * 32 + e], p[c * 32 + e + 1]);
-        }
-        tmem_st32(t_lane + cS0 + (n & 1) * 64, pk);  // P^T over the first 32 columns of this S^T buffer
-
-        ok = mbar_wait(bar_dp_full, n & 1, a.status);
-        if (!ok) break;
-        tc_fence_after();
-        uint32_t dk_[32];
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t dr[32];
-          tmem_ld32(t_lane + cDP + c * 32, dr);
+          tmem_ld32(t_lane + sbuf, sr);
           tmem_wait_ld();
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
-            const float d0 = p[c * 32 + e] * (__uint_as_float(dr[e]) - dlt[c * 32 + e]);
-            const float d1 = p[c * 32 + e + 1] * (__uint_as_float(dr[e + 1]) - dlt[c * 32 + e + 1]);
-            dk_[c * 16 + e / 2] = pack_bf16(d0, d1);
+            const float2 x = fma2(make_float2(__uint_as_float(sr[e]), __uint_as_float(sr[e + 1])), sc2,
+                                  make_float2(-lse2[e], -lse2[e + 1]));
+            p[e] = ex2(x.x);
+            p[e + 1] = ex2(x.y);
           }
-        }
-        tmem_st32(t_lane + cDP, dk_);  // dS^T over the first 32 columns of dP^T
-        // dS^T also to shared memory (row r = 128 B = 8 chunks, 128B swizzle) for the dQ^T product
-        uint8_t* ds_row = sDS + (n & 1) * SM::kDS + r * 128;
+          if (!full) {
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch)
-          *reinterpret_cast<uint4*>(ds_row + ((ch ^ (r & 7)) << 4)) =
-              make_uint4(dk_[ch * 4], dk_[ch * 4 + 1], dk_[ch * 4 + 2], dk_[ch * 4 + 3]);
+            for (int e = 0; e < 32; ++e)
+              if (!((mk >> e) & 1u)) p[e] = 0.f;
+          }
+          uint32_t pk[16];
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) pk[e / 2] = pack_bf16(p[e], p[e + 1]);
+          tmem_st16(t_lane + sbuf, pk);
+        }
+        ok = mbar_wait(bar_dp_full, n & 1, a.status);
+        if (!ok) break;
+        tc_fence_after();
+        {
+          uint32_t dr[32], dsp[16];
+          tmem_ld32(t_lane + cDP + half * 32, dr);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            const float2 y = add2(make_float2(__uint_as_float(dr[e]), __uint_as_float(dr[e + 1])),
+                                  make_float2(-dlt[e], -dlt[e + 1]));
+            const float2 z = mul2(make_float2(p[e], p[e + 1]), y);
+            dsp[e / 2] = pack_bf16(z.x, z.y);
+          }
+          tmem_st16(t_lane + cDP + half * 32, dsp);  // dS^T over the first 16 columns of this half of dP^T
+          // dS^T also to shared memory (row r = 128 B = 8 chunks, 128B swizzle) for the dQ^T product
+          uint8_t* ds_row = sDS + (n & 1) * SM::kDS + r * 128;
+#pragma unroll
+          for (int ch = 0; ch < 4; ++ch)
+            *reinterpret_cast<uint4*>(ds_row + (((half * 4 + ch) ^ (r & 7)) << 4)) =
+                make_uint4(dsp[ch * 4], dsp[ch * 4 + 1], dsp[ch * 4 + 2], dsp[ch * 4 + 3]);
+        }
         tmem_wait_st();
         tc_fence_before();
         fence_proxy_async_smem();
         mbar_arrive(bar_pds_ready);
       }
-    } else {
-      // ================= dQ drain warpgroup: one d column of dQ^T per thread =================
+    } else if (warp >= 12) {
+      // ======== dQ drain warpgroup: one d column of dQ^T per thread; TMEM -> shared -> bulk reduce-add ========
       const int d = (warp & 3) * 32 + lane;
       const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+      const bool issuer = (d == 0);
       for (int n = 0; n < N && ok; ++n) {
         const int g = n / cnt, i = cowa_bwd_tile_at(rg, n % cnt);
         const int bhq = b * a.Hq + hk * a.G + g, q0 = i * BQS;
         ok = mbar_wait(bar_dq_full, n & 1, a.status);
         if (!ok) break;
         tc_fence_after();
-        uint32_t v0[32], v1[32];
-        tmem_ld32(t_lane + cDQ, v0);
-        tmem_ld32(t_lane + cDQ + 32, v1);
+        uint32_t v[2][32];
+        tmem_ld32(t_lane + cDQ, v[0]);
+        tmem_ld32(t_lane + cDQ + 32, v[1]);
         tmem_wait_ld();
         tc_fence_before();
         mbar_arrive(bar_dq_free);
-        if (d < D) {
-          float* dst = a.dq_acc + ((size_t)bhq * a.Tpad + q0) * D + d;
-          const int nrow = min(BQS, a.Nq - q0);
 #pragma unroll
-          for (int c = 0; c < 32; ++c)
-            if (c < nrow) red_add_f32(dst + (size_t)c * D, __uint_as_float(v0[c]) * a.scale);
+        for (int hf = 0; hf < 2; ++hf) {
+          if (issuer) tma_wait_group_read<0>();  // the previous reduction has finished reading the staging tile
+          wg_sync(3);
+          if (d < D) {
 #pragma unroll
-          for (int c = 0; c < 32; ++c)
-            if (c + 32 < nrow) red_add_f32(dst + (size_t)(c + 32) * D, __uint_as_float(v1[c]) * a.scale);
+            for (int c = 0; c < 32; ++c) sDQ[c * D + d] = __uint_as_float(v[hf][c]) * a.scale;
+          }
+          fence_proxy_async_smem();
+          wg_sync(3);
+          if (issuer) {
+            tma_reduce_add_3d(&tmdQ, sDQ, 0, q0 + hf * 32, bhq);
+            tma_commit_group();
+          }
         }
       }
+      if (issuer) tma_wait_group<0>();
     }
   }
 
   // ---- epilogue: dK (compute warpgroup) and dV (drain warpgroup) -> bf16 -> shared -> TMA store ----
-  if (warp >= 2) {
-    const bool is_dk = warp < 6;
+  if ((warp >= 4 && warp < 8) || warp >= 12) {
+    const bool is_dk = warp < 8;
     const int r = (warp & 3) * 32 + lane;
     const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
     if (N > 0) ok = mbar_wait(bar_done, 0, a.status) && ok;
@@ -474,8 +496,9 @@ int launch_bwd(const void* q, const void* k, const void* v, const void* o, const
         static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse, lse2, delta, T, Tpad, BH);
     COWA_CUDA_TRY(cudaGetLastError());
   }
-  CUtensorMap mq, mk, mv, mdo, mdk, mdv;
+  CUtensorMap mq, mk, mv, mdo, mdk, mdv, mdq;
   int rc;
+  if ((rc = cowa::make_tensor_map_3d(&mdq, dq_acc, cowa::MapType::F32, D, Tpad, BH, D, 32, false))) return rc;
   if ((rc = cowa::make_tensor_map_3d(&mq, q, cowa::MapType::BF16, D, T, BH, 64, BQS))) return rc;
   if ((rc = cowa::make_tensor_map_3d(&mdo, d_o, cowa::MapType::BF16, D, T, BH, 64, BQS))) return rc;
   if ((rc = cowa::make_tensor_map_3d(&mk, k, cowa::MapType::BF16, D, T, (long long)B * Hkv, 64, BKV))) return rc;
@@ -490,11 +513,16 @@ int launch_bwd(const void* q, const void* k, const void* v, const void* o, const
   a.scale = p->softmax_scale;
   a.scale_log2 = p->softmax_scale * 1.4426950408889634f;
   a.wins = hw;
+  a.sink_tiles = 0;
+  for (int h = 0; h < Hkv; ++h) {
+    const int sk = hw.w[h].s < T ? hw.w[h].s : T;
+    a.sink_tiles = std::max(a.sink_tiles, (sk + BKV - 1) / BKV);
+  }
   COWA_CUDA_TRY(cudaFuncSetAttribute(cowa_bwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      BwdSmem<D>::kBytes));
   const long long nblocks = (long long)((T + BKV - 1) / BKV) * B * Hkv;
   if (nblocks > 0x7FFFFFFFll) return COWA_ERR_UNSUPPORTED;
-  cowa_bwd_kernel<D><<<(unsigned)nblocks, 320, BwdSmem<D>::kBytes, st>>>(mq, mk, mv, mdo, mdk, mdv, a);
+  cowa_bwd_kernel<D><<<(unsigned)nblocks, 512, BwdSmem<D>::kBytes, st>>>(mq, mk, mv, mdo, mdk, mdv, mdq, a);
   COWA_CUDA_TRY(cudaGetLastError());
   {
     const long long threads = BH * T * (D / 8);

@@ -182,35 +182,41 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         mask[c] = row_valid ? mk : 0u;
       }
     }
-    float mx = -INFINITY;
+    // row max: four independent chains of 3-input max
+    float mxa[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-    for (int c = 0; c < 4; ++c)
+    for (int c = 0; c < 4; ++c) {
+      if (!full) {
 #pragma unroll
-      for (int e = 0; e < 32; ++e) {
-        float s = __uint_as_float(sr[c][e]);
-        if (!full) s = (mask[c] >> e) & 1u ? s : -INFINITY;
-        sr[c][e] = __float_as_uint(s);
-        mx = fmaxf(mx, s);
+        for (int e = 0; e < 32; ++e)
+          if (!((mask[c] >> e) & 1u)) sr[c][e] = 0xFF800000u;  // -inf
       }
-    mx *= a.scale_log2;
+#pragma unroll
+      for (int e = 0; e < 32; e += 2)
+        mxa[(e >> 1) & 3] = max3(mxa[(e >> 1) & 3], __uint_as_float(sr[c][e]), __uint_as_float(sr[c][e + 1]));
+    }
+    const float mx = fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3])) * a.scale_log2;
     float m_new = m_ref;
     if (mx > m_ref + 8.f) m_new = mx;
     const float alpha = (m_new == m_ref) ? 1.f : ex2(m_ref - m_new);
     const float sub = (m_new == -INFINITY) ? 0.f : m_new;
     m_ref = m_new;
 
-    float rs = 0.f;
+    // p = 2^(s * scale - m): packed fp32 pairs for the multiply-add and the row sum
+    const float2 sc2 = make_float2(a.scale_log2, a.scale_log2), nsub2 = make_float2(-sub, -sub);
+    float2 rsa[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
     uint32_t pk[64];
 #pragma unroll
     for (int c = 0; c < 4; ++c)
 #pragma unroll
       for (int e = 0; e < 32; e += 2) {
-        const float p0 = ex2(fmaf(__uint_as_float(sr[c][e]), a.scale_log2, -sub));
-        const float p1 = ex2(fmaf(__uint_as_float(sr[c][e + 1]), a.scale_log2, -sub));
-        rs += p0 + p1;
-        pk[c * 16 + e / 2] = pack_bf16(p0, p1);
+        const float2 x = fma2(make_float2(__uint_as_float(sr[c][e]), __uint_as_float(sr[c][e + 1])), sc2, nsub2);
+        const float2 pp = make_float2(ex2(x.x), ex2(x.y));
+        rsa[(e >> 1) & 3] = add2(rsa[(e >> 1) & 3], pp);
+        pk[c * 16 + e / 2] = pack_bf16(pp.x, pp.y);
       }
-    l_sum = l_sum * alpha + rs;
+    const float2 rs2 = add2(add2(rsa[0], rsa[1]), add2(rsa[2], rsa[3]));
+    l_sum = l_sum * alpha + (rs2.x + rs2.y);
 
     // P over S's first 64 columns
 #pragma unroll
@@ -224,7 +230,10 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         tmem_ld32(t_O + c * 32, ov);
         tmem_wait_ld();
 #pragma unroll
-        for (int e = 0; e < 32; ++e) ov[e] = __float_as_uint(__uint_as_float(ov[e]) * alpha);
+        for (int e = 0; e < 32; e += 2) {
+          const float2 y = mul2(make_float2(__uint_as_float(ov[e]), __uint_as_float(ov[e + 1])), make_float2(alpha, alpha));
+          ov[e] = __float_as_uint(y.x); ov[e + 1] = __float_as_uint(y.y);
+        }
         tmem_st32(t_O + c * 32, ov);
       }
     }

@@ -22,7 +22,7 @@ EncodeTiledFn encode_fn() {
 }  // namespace
 
 int make_tensor_map_3d(CUtensorMap* map, const void* base, MapType type, int D, int T, long long BH, int box_d,
-                       int box_t) {
+                       int box_t, bool swizzle128) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return record_cuda_error(cudaErrorNotSupported);
   const size_t es = type == MapType::BF16 ? 2 : 4;
@@ -32,7 +32,7 @@ int make_tensor_map_3d(CUtensorMap* map, const void* base, MapType type, int D, 
   cuuint32_t estr[3] = {1, 1, 1};
   CUresult r = fn(map, type == MapType::BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
                   3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return record_cuda_error(cudaErrorInvalidValue);
   return COWA_OK;
