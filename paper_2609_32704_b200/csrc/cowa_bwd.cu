@@ -93,7 +93,7 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   constexpr int SLAB_KV = BKV * 128;  // bytes of one 64-wide slab of a 128-row tile
   constexpr int SLAB_QS = BQS * 128;  // ... of a 64-row tile
   // TMEM columns
-  constexpr uint32_t cS0 = 0, cDP = 128, cDQ = 192, cDK = 256, cDV = 384, TMEM_COLS = 512;
+  constexpr uint32_t cS0 = 0, cDP0 = 128, cDK = 256, cDV = 384, TMEM_COLS = 512;  // S^T x2, dP^T/dQ^T x2, dK, dV
   constexpr uint32_t ID_ST = idesc_bf16(128, BQS, 0, 0);   // S^T, dP^T
   constexpr uint32_t ID_ACC = idesc_bf16(128, D, 0, 1);    // dV, dK (B = dO / Q, MN-major)
   constexpr uint32_t ID_DQ = idesc_bf16(128, BQS, 1, 1);   // dQ^T (A = K^T, B = dS^T, both MN-major)
@@ -108,15 +108,16 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   float* sDQ = reinterpret_cast<float*>(smem + SM::oDQ);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::oBar);
   uint64_t* bar_kv = bars + 0;
-  uint64_t* bar_ld_full = bars + 1;             // [NST]
-  uint64_t* bar_ld_empty = bars + 1 + NST;      // [NST]
-  uint64_t* bar_s_full = bars + 1 + 2 * NST;    // [2]
-  uint64_t* bar_dp_full = bars + 3 + 2 * NST;
-  uint64_t* bar_pds_ready = bars + 4 + 2 * NST; // count 256
-  uint64_t* bar_dq_full = bars + 5 + 2 * NST;
-  uint64_t* bar_dq_free = bars + 6 + 2 * NST;   // count 128
-  uint64_t* bar_done = bars + 7 + 2 * NST;
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 8 + 2 * NST);
+  uint64_t* bar_ld_full = bars + 1;             // [NST]  Q/dO/LSE/Delta of a step have landed
+  uint64_t* bar_ld_empty = bars + 1 + NST;      // [NST]  the step's products have consumed the stage
+  uint64_t* bar_s_full = bars + 1 + 2 * NST;    // [2]    S^T of a step is in TMEM buffer b
+  uint64_t* bar_dp_full = bars + 3 + 2 * NST;   // [2]    dP^T ...
+  uint64_t* bar_p_ready = bars + 5 + 2 * NST;   // [2]    count 128: P^T written over S^T
+  uint64_t* bar_ds_ready = bars + 7 + 2 * NST;  // [2]    count 128: dS^T in TMEM and shared memory, dP^T consumed
+  uint64_t* bar_dq_full = bars + 9 + 2 * NST;   // [2]    dQ^T is in the columns dP^T left
+  uint64_t* bar_dq_free = bars + 11 + 2 * NST;  // [2]    count 128: dQ^T drained
+  uint64_t* bar_done = bars + 13 + 2 * NST;
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 14 + 2 * NST);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -145,9 +146,12 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   if (tid == 0) {
     mbar_init(bar_kv, 1);
     for (int s = 0; s < NST; ++s) { mbar_init(bar_ld_full + s, 1); mbar_init(bar_ld_empty + s, 1); }
-    mbar_init(bar_s_full, 1); mbar_init(bar_s_full + 1, 1);
-    mbar_init(bar_dp_full, 1); mbar_init(bar_pds_ready, 256);
-    mbar_init(bar_dq_full, 1); mbar_init(bar_dq_free, 128); mbar_init(bar_done, 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(bar_s_full + s, 1); mbar_init(bar_dp_full + s, 1);
+      mbar_init(bar_p_ready + s, 128); mbar_init(bar_ds_ready + s, 128);
+      mbar_init(bar_dq_full + s, 1); mbar_init(bar_dq_free + s, 128);
+    }
+    mbar_init(bar_done, 1);
     fence_mbar_init();
   }
   if (warp == 0) {
@@ -162,225 +166,9 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 
   bool ok = true;
 
-  if (N > 0) {
-    if (warp == 0) {
-      // ================= TMA producer =================
-      if (lane == 0) {
-        prefetch_tmap(&tmQ); prefetch_tmap(&tmdO); prefetch_tmap(&tmK); prefetch_tmap(&tmV);
-        mbar_expect_tx(bar_kv, 2 * SM::kKV);
-        for (int s = 0; s < NSLAB; ++s) {
-          tma_load_3d(sK + s * SLAB_KV, &tmK, bar_kv, s * 64, k0, bhk);
-          tma_load_3d(sV + s * SLAB_KV, &tmV, bar_kv, s * 64, k0, bhk);
-        }
-        for (int n = 0; n < N && ok; ++n) {
-          const int st = n % NST;
-          if (n >= NST) ok = mbar_wait(bar_ld_empty + st, ((n / NST) - 1) & 1, a.status);
-          if (!ok) break;
-          const int g = n / cnt, i = cowa_bwd_tile_at(rg, n % cnt);
-          const int bhq = b * a.Hq + hk * a.G + g, q0 = i * BQS;
-          uint8_t* sQ = sStage + st * SM::kStage;
-          uint8_t* sdO = sQ + SM::kQS;
-          mbar_expect_tx(bar_ld_full + st, SM::kStage + 512);
-          for (int s = 0; s < NSLAB; ++s) {
-            tma_load_3d(sQ + s * SLAB_QS, &tmQ, bar_ld_full + st, s * 64, q0, bhq);
-            tma_load_3d(sdO + s * SLAB_QS, &tmdO, bar_ld_full + st, s * 64, q0, bhq);
-          }
-          bulk_load_1d(sVec + st * 128, a.lse2 + (size_t)bhq * a.Tpad + q0, 256, bar_ld_full + st);
-          bulk_load_1d(sVec + st * 128 + 64, a.delta + (size_t)bhq * a.Tpad + q0, 256, bar_ld_full + st);
-        }
-      }
-    } else if (warp == 1) {
-      // ================= MMA issuer =================
-      if (lane == 0) {
-        auto gemm_st = [&](uint32_t d_col, const uint8_t* sA, const uint8_t* sB) {  // [128 x 64] = A[128xD] B[64xD]^T
-#pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk) {
-            const uint32_t oa = (kk / 4) * SLAB_KV + (kk % 4) * 32, ob = (kk / 4) * SLAB_QS + (kk % 4) * 32;
-            mma_ss(tmem_base + d_col, smem_desc_sw128(smem_u32(sA) + oa, 16, 1024),
-                   smem_desc_sw128(smem_u32(sB) + ob, 16, 1024), ID_ST, kk > 0);
-          }
-        };
-        auto gemm_acc = [&](uint32_t d_col, uint32_t a_col, const uint8_t* sB, bool first) {  // [128 x D] += A^T-in-TMEM B
-#pragma unroll
-          for (int kk = 0; kk < BQS / 16; ++kk)  // A: query columns 0-31 at a_col, 32-63 at a_col + 32
-            mma_ts(tmem_base + d_col, tmem_base + a_col + (kk & 1) * 8 + (kk >> 1) * 32,
-                   smem_desc_sw128(smem_u32(sB) + kk * 2048, SLAB_QS, 1024), ID_ACC, (!first || kk > 0) ? 1u : 0u);
-        };
-        auto gemm_dq = [&](const uint8_t* sB) {  // dQ^T[D x 64] = K^T dS^T
-#pragma unroll
-          for (int kk = 0; kk < BKV / 16; ++kk)
-            mma_ss(tmem_base + cDQ, smem_desc_sw128(smem_u32(sK) + kk * 2048, D == 128 ? SLAB_KV : 0, 1024),
-                   smem_desc_sw128(smem_u32(sB) + kk * 2048, 0, 1024), ID_DQ, kk > 0);
-        };
-        ok = mbar_wait(bar_kv, 0, a.status);
-        // prologue: S^T(0), dP^T(0), S^T(1)
-        ok = ok && mbar_wait(bar_ld_full + 0, 0, a.status);
-        if (ok) {
-          tc_fence_after();
-          gemm_st(cS0, sK, sStage);
-          mma_commit(bar_s_full + 0);
-          gemm_st(cDP, sV, sStage + SM::kQS);
-          mma_commit(bar_dp_full);
-        }
-        if (ok && N > 1) {
-          ok = mbar_wait(bar_ld_full + 1, 0, a.status);
-          if (ok) {
-            tc_fence_after();
-            gemm_st(cS0 + 64, sK, sStage + SM::kStage);
-            mma_commit(bar_s_full + 1);
-          }
-        }
-        for (int n = 0; n < N && ok; ++n) {
-          const int st = n % NST;
-          uint8_t* sQ = sStage + st * SM::kStage;
-          uint8_t* sdO = sQ + SM::kQS;
-          ok = mbar_wait(bar_pds_ready, n & 1, a.status);
-          if (!ok) break;
-          tc_fence_after();
-          gemm_acc(cDV, cS0 + (n & 1) * 64, sdO, n == 0);  // dV += P^T dO
-          gemm_acc(cDK, cDP, sQ, n == 0);                  // dK += dS^T Q
-          mma_commit(bar_ld_empty + st);
-          if (n + 1 < N) {                                 // dP^T(n+1): its stage was awaited one step ago
-            const int s1 = (n + 1) % NST;
-            gemm_st(cDP, sV, sStage + s1 * SM::kStage + SM::kQS);
-            mma_commit(bar_dp_full);
-          }
-          if (n + 2 < N) {                                 // S^T(n+2) into the buffer P^T(n) just left
-            const int s2 = (n + 2) % NST;
-            ok = mbar_wait(bar_ld_full + s2, ((n + 2) / NST) & 1, a.status);
-            if (!ok) break;
-            tc_fence_after();
-            gemm_st(cS0 + (n & 1) * 64, sK, sStage + s2 * SM::kStage);
-            mma_commit(bar_s_full + (n & 1));
-          }
-          if (n > 0) {
-            ok = mbar_wait(bar_dq_free, (n - 1) & 1, a.status);
-            if (!ok) break;
-            tc_fence_after();
-          }
-          gemm_dq(sDS + (n & 1) * SM::kDS);
-          mma_commit(bar_dq_full);
-        }
-        mma_commit(bar_done);
-      }
-    } else if (warp >= 4 && warp < 12) {
-      // ======== two compute warpgroups: P^T and dS^T, one KV row per thread, 32 query columns each ========
-      const int half = (warp - 4) >> 2;      // 0: query columns 0-31, 1: 32-63
-      const int r = (warp & 3) * 32 + lane;  // KV row = TMEM lane
-      const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
-      const int kcol = k0 + r;               // key index of this thread
-      const long long kpos = (long long)kcol - off;  // first causal query of this key
-      const float2 sc2 = make_float2(a.scale_log2, a.scale_log2);
-      for (int n = 0; n < N && ok; ++n) {
-        const int st = n % NST;
-        const int i = cowa_bwd_tile_at(rg, n % cnt);
-        const int q0 = i * BQS;
-        const bool full = cowa_tile_full(w, q0, BQS, k0, BKV, off, a.Nq, a.Nk);
-        uint32_t mk = 0xFFFFFFFFu;
-        if (!full) {
-          const long long qend = a.Nq - 1, base = q0 + half * 32;
-          uint32_t m = interval_bits32(kpos, min(kpos + w.n - 1, qend), base);
-          if (w.l > 0)
-            m |= interval_bits32(kpos + w.n + w.g, min(kpos + (long long)w.n + w.g + w.l - 1, qend), base);
-          if (kcol < w.s) m |= interval_bits32(kpos, qend, base);
-          mk = kcol < a.Nk ? m : 0u;
-        }
-        const float* lse2 = sVec + st * 128 + half * 32;
-        const float* dlt = sVec + st * 128 + 64 + half * 32;
-        const uint32_t sbuf = cS0 + (n & 1) * 64 + half * 32;  // this half's S^T columns; P^T goes over the first 16
-        ok = mbar_wait(bar_ld_full + st, (n / NST) & 1, a.status);
-        ok = ok && mbar_wait(bar_s_full + (n & 1), (n >> 1) & 1, a.status);
-        if (!ok) break;
-        tc_fence_after();
-        float p[32];
-        {
-          uint32_t sr[32];
-          tmem_ld32(t_lane + sbuf, sr);
-          tmem_wait_ld();
-#pragma unroll
-          for (int e = 0; e < 32; e += 2) {
-            const float2 x = fma2(make_float2(__uint_as_float(sr[e]), __uint_as_float(sr[e + 1])), sc2,
-                                  make_float2(-lse2[e], -lse2[e + 1]));
-            p[e] = ex2(x.x);
-            p[e + 1] = ex2(x.y);
-          }
-          if (!full) {
-#pragma unroll
-            for (int e = 0; e < 32; ++e)
-              if (!((mk >> e) & 1u)) p[e] = 0.f;
-          }
-          uint32_t pk[16];
-#pragma unroll
-          for (int e = 0; e < 32; e += 2) pk[e / 2] = pack_bf16(p[e], p[e + 1]);
-          tmem_st16(t_lane + sbuf, pk);
-        }
-        ok = mbar_wait(bar_dp_full, n & 1, a.status);
-        if (!ok) break;
-        tc_fence_after();
-        {
-          uint32_t dr[32], dsp[16];
-          tmem_ld32(t_lane + cDP + half * 32, dr);
-          tmem_wait_ld();
-#pragma unroll
-          for (int e = 0; e < 32; e += 2) {
-            const float2 y = add2(make_float2(__uint_as_float(dr[e]), __uint_as_float(dr[e + 1])),
-                                  make_float2(-dlt[e], -dlt[e + 1]));
-            const float2 z = mul2(make_float2(p[e], p[e + 1]), y);
-            dsp[e / 2] = pack_bf16(z.x, z.y);
-          }
-          tmem_st16(t_lane + cDP + half * 32, dsp);  // dS^T over the first 16 columns of this half of dP^T
-          // dS^T also to shared memory (row r = 128 B = 8 chunks, 128B swizzle) for the dQ^T product
-          uint8_t* ds_row = sDS + (n & 1) * SM::kDS + r * 128;
-#pragma unroll
-          for (int ch = 0; ch < 4; ++ch)
-            *reinterpret_cast<uint4*>(ds_row + (((half * 4 + ch) ^ (r & 7)) << 4)) =
-                make_uint4(dsp[ch * 4], dsp[ch * 4 + 1], dsp[ch * 4 + 2], dsp[ch * 4 + 3]);
-        }
-        tmem_wait_st();
-        tc_fence_before();
-        fence_proxy_async_smem();
-        mbar_arrive(bar_pds_ready);
-      }
-    } else if (warp >= 12) {
-      // ======== dQ drain warpgroup: one d column of dQ^T per thread; TMEM -> shared -> bulk reduce-add ========
-      const int d = (warp & 3) * 32 + lane;
-      const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
-      const bool issuer = (d == 0);
-      for (int n = 0; n < N && ok; ++n) {
-        const int g = n / cnt, i = cowa_bwd_tile_at(rg, n % cnt);
-        const int bhq = b * a.Hq + hk * a.G + g, q0 = i * BQS;
-        ok = mbar_wait(bar_dq_full, n & 1, a.status);
-        if (!ok) break;
-        tc_fence_after();
-        uint32_t v[2][32];
-        tmem_ld32(t_lane + cDQ, v[0]);
-        tmem_ld32(t_lane + cDQ + 32, v[1]);
-        tmem_wait_ld();
-        tc_fence_before();
-        mbar_arrive(bar_dq_free);
-#pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-          if (issuer) tma_wait_group_read<0>();  // the previous reduction has finished reading the staging tile
-          wg_sync(3);
-          if (d < D) {
-#pragma unroll
-            for (int c = 0; c < 32; ++c) sDQ[c * D + d] = __uint_as_float(v[hf][c]) * a.scale;
-          }
-          fence_proxy_async_smem();
-          wg_sync(3);
-          if (issuer) {
-            tma_reduce_add_3d(&tmdQ, sDQ, 0, q0 + hf * 32, bhq);
-            tma_commit_group();
-          }
-        }
-      }
-      if (issuer) tma_wait_group<0>();
-    }
-  }
-
-  // ---- epilogue: dK (compute warpgroup) and dV (drain warpgroup) -> bf16 -> shared -> TMA store ----
-  if ((warp >= 4 && warp < 8) || warp >= 12) {
-    const bool is_dk = warp < 8;
+  // dK (first compute warpgroup) and dV (drain warpgroup): TMEM -> bf16 -> shared -> TMA store.  Called from
+  // inside the role branches so that it is compiled under that role's register budget.
+  auto store_grad = [&](bool is_dk) {
     const int r = (warp & 3) * 32 + lane;
     const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
     if (N > 0) ok = mbar_wait(bar_done, 0, a.status) && ok;
@@ -415,6 +203,256 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       for (int s = 0; s < NSLAB; ++s) tma_store_3d(is_dk ? &tmdK : &tmdV, sOut + s * SLAB_KV, s * 64, k0, bhk);
       tma_commit_group();
       tma_wait_group<0>();
+    }
+  };
+
+  // Register budget per role: 128 per thread at launch (512 threads), moved to where the work is.  Each
+  // setmaxnreg sits at the top of its own branch so that the code below it is compiled for that budget.
+  if (warp < 4) {
+    setmaxnreg_dec<64>();
+    if (warp == 0) {
+      // ================= TMA producer =================
+      if (lane == 0 && N > 0) {
+        prefetch_tmap(&tmQ); prefetch_tmap(&tmdO); prefetch_tmap(&tmK); prefetch_tmap(&tmV);
+        mbar_expect_tx(bar_kv, 2 * SM::kKV);
+        for (int s = 0; s < NSLAB; ++s) {
+          tma_load_3d(sK + s * SLAB_KV, &tmK, bar_kv, s * 64, k0, bhk);
+          tma_load_3d(sV + s * SLAB_KV, &tmV, bar_kv, s * 64, k0, bhk);
+        }
+        for (int n = 0; n < N && ok; ++n) {
+          const int st = n % NST;
+          if (n >= NST) ok = mbar_wait(bar_ld_empty + st, ((n / NST) - 1) & 1, a.status);
+          if (!ok) break;
+          const int g = n / cnt, i = cowa_bwd_tile_at(rg, n % cnt);
+          const int bhq = b * a.Hq + hk * a.G + g, q0 = i * BQS;
+          uint8_t* sQ = sStage + st * SM::kStage;
+          uint8_t* sdO = sQ + SM::kQS;
+          mbar_expect_tx(bar_ld_full + st, SM::kStage + 512);
+          for (int s = 0; s < NSLAB; ++s) {
+            tma_load_3d(sQ + s * SLAB_QS, &tmQ, bar_ld_full + st, s * 64, q0, bhq);
+            tma_load_3d(sdO + s * SLAB_QS, &tmdO, bar_ld_full + st, s * 64, q0, bhq);
+          }
+          bulk_load_1d(sVec + st * 128, a.lse2 + (size_t)bhq * a.Tpad + q0, 256, bar_ld_full + st);
+          bulk_load_1d(sVec + st * 128 + 64, a.delta + (size_t)bhq * a.Tpad + q0, 256, bar_ld_full + st);
+        }
+      }
+    } else if (warp == 1) {
+      // ================= MMA issuer =================
+      if (lane == 0 && N > 0) {
+        // Descriptors are built once per operand base; a byte offset o inside the tile is added as o >> 4
+        // to the descriptor's address field (the tiles never cross the field's range).
+        const uint64_t dK_k = smem_desc_sw128(smem_u32(sK), 16, 1024);                           // K, K-major (A of S^T)
+        const uint64_t dV_k = smem_desc_sw128(smem_u32(sV), 16, 1024);                           // V, K-major (A of dP^T)
+        const uint64_t dK_mn = smem_desc_sw128(smem_u32(sK), D == 128 ? SLAB_KV : 0, 1024);      // K^T, MN-major (A of dQ^T)
+        auto gemm_st = [&](uint32_t d_col, uint64_t dA, const uint8_t* sB) {  // [128 x 64] = A[128xD] B[64xD]^T
+          const uint64_t dB = smem_desc_sw128(smem_u32(sB), 16, 1024);
+#pragma unroll
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint32_t oa = (kk / 4) * SLAB_KV + (kk % 4) * 32, ob = (kk / 4) * SLAB_QS + (kk % 4) * 32;
+            mma_ss(tmem_base + d_col, dA + (oa >> 4), dB + (ob >> 4), ID_ST, kk > 0);
+          }
+        };
+        auto gemm_acc = [&](uint32_t d_col, uint32_t a_col, const uint8_t* sB, bool first) {  // [128 x D] += A^T-in-TMEM B
+          const uint64_t dB = smem_desc_sw128(smem_u32(sB), SLAB_QS, 1024);
+#pragma unroll
+          for (int kk = 0; kk < BQS / 16; ++kk)
+            mma_ts(tmem_base + d_col, tmem_base + a_col + kk * 8, dB + ((kk * 2048) >> 4), ID_ACC,
+                   (!first || kk > 0) ? 1u : 0u);
+        };
+        auto gemm_dq = [&](uint32_t d_col, const uint8_t* sB) {  // dQ^T[D x 64] = K^T dS^T
+          const uint64_t dB = smem_desc_sw128(smem_u32(sB), 0, 1024);
+#pragma unroll
+          for (int kk = 0; kk < BKV / 16; ++kk)
+            mma_ss(tmem_base + d_col, dK_mn + ((kk * 2048) >> 4), dB + ((kk * 2048) >> 4), ID_DQ, kk > 0);
+        };
+        ok = mbar_wait(bar_kv, 0, a.status);
+        // prologue: S^T(0), dP^T(0), S^T(1)
+        ok = ok && mbar_wait(bar_ld_full + 0, 0, a.status);
+        if (ok) {
+          tc_fence_after();
+          gemm_st(cS0, dK_k, sStage);
+          mma_commit(bar_s_full + 0);
+          gemm_st(cDP0, dV_k, sStage + SM::kQS);
+          mma_commit(bar_dp_full + 0);
+        }
+        if (ok && N > 1) {
+          ok = mbar_wait(bar_ld_full + 1, 0, a.status);
+          if (ok) {
+            tc_fence_after();
+            gemm_st(cS0 + 64, dK_k, sStage + SM::kStage);
+            mma_commit(bar_s_full + 1);
+          }
+        }
+        // Step n uses TMEM buffer b = n & 1 (the two compute warpgroups alternate steps).  Issue order:
+        //   dV(n) | dP^T(n+1) | dK(n) | dQ^T(n) | S^T(n+2)
+        // so that every wait below is for something produced about one step earlier.
+        for (int n = 0; n < N && ok; ++n) {
+          const int st = n % NST, b_ = n & 1;
+          const uint32_t par = (n >> 1) & 1;
+          uint8_t* sQ = sStage + st * SM::kStage;
+          uint8_t* sdO = sQ + SM::kQS;
+          const uint32_t sbuf = cS0 + b_ * 64, dpbuf = cDP0 + b_ * 64;
+          ok = mbar_wait(bar_p_ready + b_, par, a.status);
+          if (!ok) break;
+          tc_fence_after();
+          gemm_acc(cDV, sbuf, sdO, n == 0);                // dV += P^T dO
+          if (n + 1 < N) {                                 // dP^T(n+1) into the other buffer, once dQ^T(n-1) has left it
+            if (n >= 1) {
+              ok = mbar_wait(bar_dq_free + (b_ ^ 1), ((n - 1) >> 1) & 1, a.status);
+              if (!ok) break;
+              tc_fence_after();
+            }
+            gemm_st(cDP0 + (b_ ^ 1) * 64, dV_k, sStage + ((n + 1) % NST) * SM::kStage + SM::kQS);
+            mma_commit(bar_dp_full + (b_ ^ 1));
+          }
+          ok = mbar_wait(bar_ds_ready + b_, par, a.status);
+          if (!ok) break;
+          tc_fence_after();
+          gemm_acc(cDK, sbuf + 32, sQ, n == 0);            // dK += dS^T Q
+          mma_commit(bar_ld_empty + st);
+          gemm_dq(dpbuf, sDS + b_ * SM::kDS);              // dQ^T = K^T dS^T, over the consumed dP^T(n)
+          mma_commit(bar_dq_full + b_);
+          if (n + 2 < N) {                                 // S^T(n+2) into the buffer that P^T(n), dS^T(n) just left
+            const int s2 = (n + 2) % NST;
+            ok = mbar_wait(bar_ld_full + s2, ((n + 2) / NST) & 1, a.status);
+            if (!ok) break;
+            tc_fence_after();
+            gemm_st(sbuf, dK_k, sStage + s2 * SM::kStage);
+            mma_commit(bar_s_full + b_);
+          }
+        }
+        mma_commit(bar_done);
+      }
+    }
+  } else if (warp < 12) {
+    setmaxnreg_inc<176>();
+    {
+      // ======== two compute warpgroups alternate steps: P^T and dS^T, one KV row per thread ========
+      const int wg = (warp - 4) >> 2;        // steps n with n & 1 == wg, TMEM buffer wg
+      const int r = (warp & 3) * 32 + lane;  // KV row = TMEM lane
+      const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+      const uint32_t sbuf = t_lane + cS0 + wg * 64, dpbuf = t_lane + cDP0 + wg * 64;
+      const int kcol = k0 + r;               // key index of this thread
+      const long long kpos = (long long)kcol - off;  // first causal query of this key
+      const float2 sc2 = make_float2(a.scale_log2, a.scale_log2);
+      uint8_t* ds_row = sDS + wg * SM::kDS + r * 128;
+      for (int n = wg; n < N && ok; n += 2) {
+        const int st = n % NST;
+        const uint32_t par = (n >> 1) & 1;
+        const int i = cowa_bwd_tile_at(rg, n % cnt);
+        const int q0 = i * BQS;
+        const bool full = cowa_tile_full(w, q0, BQS, k0, BKV, off, a.Nq, a.Nk);
+        uint32_t mk[2] = {0xFFFFFFFFu, 0xFFFFFFFFu};
+        if (!full) {
+          const long long qend = a.Nq - 1;
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {
+            const long long base = q0 + c * 32;
+            uint32_t m = interval_bits32(kpos, min(kpos + w.n - 1, qend), base);
+            if (w.l > 0)
+              m |= interval_bits32(kpos + w.n + w.g, min(kpos + (long long)w.n + w.g + w.l - 1, qend), base);
+            if (kcol < w.s) m |= interval_bits32(kpos, qend, base);
+            mk[c] = kcol < a.Nk ? m : 0u;
+          }
+        }
+        const float* lse2 = sVec + st * 128;
+        const float* dlt = lse2 + 64;
+        ok = mbar_wait(bar_ld_full + st, (n / NST) & 1, a.status);
+        ok = ok && mbar_wait(bar_s_full + wg, par, a.status);
+        if (!ok) break;
+        tc_fence_after();
+        float p[64];
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t sr[32], pk[16];
+          tmem_ld32(sbuf + c * 32, sr);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            const float2 x = fma2(make_float2(__uint_as_float(sr[e]), __uint_as_float(sr[e + 1])), sc2,
+                                  make_float2(-lse2[c * 32 + e], -lse2[c * 32 + e + 1]));
+            p[c * 32 + e] = ex2(x.x);
+            p[c * 32 + e + 1] = ex2(x.y);
+          }
+          if (!full) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e)
+              if (!((mk[c] >> e) & 1u)) p[c * 32 + e] = 0.f;
+          }
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) pk[e / 2] = pack_bf16(p[c * 32 + e], p[c * 32 + e + 1]);
+          tmem_st16(sbuf + c * 16, pk);  // P^T: 64 queries packed into columns 0-31 of this S^T buffer
+        }
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar_p_ready + wg);
+
+        ok = mbar_wait(bar_dp_full + wg, par, a.status);
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t dr[32], dsp[16];
+          tmem_ld32(dpbuf + c * 32, dr);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            const float2 y = add2(make_float2(__uint_as_float(dr[e]), __uint_as_float(dr[e + 1])),
+                                  make_float2(-dlt[c * 32 + e], -dlt[c * 32 + e + 1]));
+            const float2 z = mul2(make_float2(p[c * 32 + e], p[c * 32 + e + 1]), y);
+            dsp[e / 2] = pack_bf16(z.x, z.y);
+          }
+          tmem_st16(sbuf + 32 + c * 16, dsp);  // dS^T beside P^T, in columns 32-63 of the S^T buffer
+          // dS^T also to shared memory (row r = 128 B = 8 chunks, 128B swizzle) for the dQ^T product
+#pragma unroll
+          for (int ch = 0; ch < 4; ++ch)
+            *reinterpret_cast<uint4*>(ds_row + (((c * 4 + ch) ^ (r & 7)) << 4)) =
+                make_uint4(dsp[ch * 4], dsp[ch * 4 + 1], dsp[ch * 4 + 2], dsp[ch * 4 + 3]);
+        }
+        tmem_wait_st();
+        tc_fence_before();
+        fence_proxy_async_smem();
+        mbar_arrive(bar_ds_ready + wg);
+      }
+      if (wg == 0) store_grad(true);
+    }
+  } else {
+    setmaxnreg_dec<96>();
+    {
+      // ======== dQ drain warpgroup: one d column of dQ^T per thread; TMEM -> shared -> bulk reduce-add ========
+      const int d = (warp & 3) * 32 + lane;
+      const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+      const bool issuer = (d == 0);
+      for (int n = 0; n < N && ok; ++n) {
+        const int g = n / cnt, i = cowa_bwd_tile_at(rg, n % cnt);
+        const int bhq = b * a.Hq + hk * a.G + g, q0 = i * BQS;
+        ok = mbar_wait(bar_dq_full + (n & 1), (n >> 1) & 1, a.status);
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t v[2][32];
+        tmem_ld32(t_lane + cDP0 + (n & 1) * 64, v[0]);
+        tmem_ld32(t_lane + cDP0 + (n & 1) * 64 + 32, v[1]);
+        tmem_wait_ld();
+        tc_fence_before();
+        mbar_arrive(bar_dq_free + (n & 1));
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          if (issuer) tma_wait_group_read<0>();  // the previous reduction has finished reading the staging tile
+          wg_sync(3);
+          if (d < D) {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) sDQ[c * D + d] = __uint_as_float(v[hf][c]) * a.scale;
+          }
+          fence_proxy_async_smem();
+          wg_sync(3);
+          if (issuer) {
+            tma_reduce_add_3d(&tmdQ, sDQ, 0, q0 + hf * 32, bhq);
+            tma_commit_group();
+          }
+        }
+      }
+      if (issuer) tma_wait_group<0>();
+      store_grad(false);
     }
   }
 
