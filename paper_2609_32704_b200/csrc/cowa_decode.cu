@@ -89,7 +89,10 @@ __device__ __forceinline__ float bf16lo(uint32_t x) { return __uint_as_float(x <
 __device__ __forceinline__ float bf16hi(uint32_t x) { return __uint_as_float(x & 0xffff0000u); }
 
 template <int D, int G>
-__global__ void __launch_bounds__(kThreads) cowa_decode_split_kernel(const DecodeArgs a) {
+#ifndef COWA_DEC_MINB
+#define COWA_DEC_MINB 7
+#endif
+__global__ void __launch_bounds__(kThreads, COWA_DEC_MINB) cowa_decode_split_kernel(const DecodeArgs a) {
   static_assert(D == 64 || D == 128, "head dim");
   static_assert(G >= 1 && G <= 8, "group size per mma n-tile");
   constexpr int DC = D / 8;           // 16-byte slices per row
@@ -203,7 +206,10 @@ __global__ void __launch_bounds__(kThreads) cowa_decode_split_kernel(const Decod
 #pragma unroll
     for (int i = 0; i < 8; ++i) acc[h][i] = 0.f;
 
-  constexpr int U = 4;
+#ifndef COWA_DEC_U
+#define COWA_DEC_U 4
+#endif
+  constexpr int U = COWA_DEC_U;
   for (int r0 = rs; r0 < clen; r0 += RP * U) {
     uint4 vv[U];
 #pragma unroll
@@ -248,29 +254,81 @@ __global__ void __launch_bounds__(kThreads) cowa_decode_split_kernel(const Decod
 }
 
 // Merge of the split states: M = max m_s, L = sum l_s 2^(m_s - M), o = sum o_s 2^(m_s - M) / L,
-// lse = ln2 * (M + log2 L).  One block per (sequence, QO head), D threads.
+// lse = ln2 * (M + log2 L).  One block of 4 warps per (sequence, QO head): every warp reduces M and L
+// with shuffles, takes every fourth split with D/32 columns per lane (several loads in flight), and the
+// four partial sums meet in shared memory.
 template <int D>
-__global__ void __launch_bounds__(D) cowa_decode_combine_kernel(const float* __restrict__ ws_o,
-                                                                const float* __restrict__ ws_m,
-                                                                const float* __restrict__ ws_l,
-                                                                __nv_bfloat16* __restrict__ o,
-                                                                float* __restrict__ lse, int S) {
+__global__ void __launch_bounds__(128) cowa_decode_combine_kernel(const float* __restrict__ ws_o,
+                                                                  const float* __restrict__ ws_m,
+                                                                  const float* __restrict__ ws_l,
+                                                                  __nv_bfloat16* __restrict__ o,
+                                                                  float* __restrict__ lse, int S) {
+  constexpr int V = D / 32;  // columns per lane
+  __shared__ float part[4][D];
   const size_t bh = blockIdx.x;
-  const int tid = threadIdx.x, lane = tid & 31;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const float* m = ws_m + bh * S;
   const float* l = ws_l + bh * S;
-  float mx = -INFINITY;
-  for (int s = lane; s < S; s += 32) mx = fmaxf(mx, m[s]);
+  const float* po = ws_o + bh * S * D + lane * V;
+  float acc[V];
 #pragma unroll
-  for (int o_ = 16; o_ > 0; o_ >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o_));
-  float L = 0.f;
-  for (int s = lane; s < S; s += 32) L += l[s] * exp2f(m[s] - mx);  // empty splits: l = 0, m = -inf -> 0
+  for (int i = 0; i < V; ++i) acc[i] = 0.f;
+  float mx = -INFINITY, L = 0.f;
+  constexpr int U = 8;
+  if (S <= 32) {
+    // one round trip: every load is issued before the first use
+    const float ms = lane < S ? m[lane] : -INFINITY;
+    const float ls = lane < S ? l[lane] : 0.f;
+    float x[U][V];
 #pragma unroll
-  for (int o_ = 16; o_ > 0; o_ >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o_);
-  float acc = 0.f;
-  const float* po = ws_o + bh * S * D + tid;
-  for (int s = 0; s < S; ++s) acc = fmaf(po[(size_t)s * D], exp2f(m[s] - mx), acc);
-  o[bh * D + tid] = __float2bfloat16_rn(acc / L);
+    for (int u = 0; u < U; ++u) {
+      const int s = warp + 4 * u;
+#pragma unroll
+      for (int i = 0; i < V; ++i) x[u][i] = s < S ? po[(size_t)s * D + i] : 0.f;
+    }
+    mx = ms;
+#pragma unroll
+    for (int o_ = 16; o_ > 0; o_ >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o_));
+    const float wl = exp2f(ms - mx);  // empty splits: m = -inf -> weight 0
+    L = ls * wl;
+#pragma unroll
+    for (int o_ = 16; o_ > 0; o_ >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o_);
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const float wgt = __shfl_sync(0xffffffffu, wl, (warp + 4 * u) & 31);
+#pragma unroll
+      for (int i = 0; i < V; ++i) acc[i] = fmaf(x[u][i], wgt, acc[i]);
+    }
+  } else {
+    for (int s = lane; s < S; s += 32) mx = fmaxf(mx, m[s]);
+#pragma unroll
+    for (int o_ = 16; o_ > 0; o_ >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o_));
+    for (int s = lane; s < S; s += 32) L += l[s] * exp2f(m[s] - mx);
+#pragma unroll
+    for (int o_ = 16; o_ > 0; o_ >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o_);
+    for (int s0 = warp; s0 < S; s0 += 4 * U) {
+      float x[U][V], wgt[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int s = s0 + 4 * u;
+        const bool in = s < S;
+        wgt[u] = in ? exp2f(m[s] - mx) : 0.f;
+#pragma unroll
+        for (int i = 0; i < V; ++i) x[u][i] = in ? po[(size_t)s * D + i] : 0.f;
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u)
+#pragma unroll
+        for (int i = 0; i < V; ++i) acc[i] = fmaf(x[u][i], wgt[u], acc[i]);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < V; ++i) part[warp][lane * V + i] = acc[i];
+  __syncthreads();
+  if (tid < D) {
+    const float v = (part[0][tid] + part[1][tid]) + (part[2][tid] + part[3][tid]);
+    o[bh * D + tid] = __float2bfloat16_rn(v / L);
+  }
   if (lse && tid == 0) lse[bh] = 0.6931471805599453f * (mx + log2f(L));
 }
 
@@ -284,14 +342,48 @@ int max_visible(int Tmax, int hg, const cowa_params_t* p) {
   return (int)(v < Tmax ? v : Tmax);
 }
 
-int pick_splits(int B, int Tmax, int Hkv, const cowa_params_t* p) {
+// Blocks of the split kernel that fit the current device at once (SM count x resident blocks per SM).
+// Falls back to 148 x 7 (B200, 72 registers, 16 KB shared memory) when no device can be queried.
+template <int D, int G>
+int resident_blocks_of() {
+  int dev = 0, sms = 0, occ = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, cowa_decode_split_kernel<D, G>, kThreads, 0) != cudaSuccess)
+    return 0;
+  return sms * occ;
+}
+
+int resident_blocks(int D, int G) {
+  static int cache[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};
+  const int di = D == 128 ? 1 : 0, gi = G == 1 ? 0 : G == 2 ? 1 : G == 4 ? 2 : 3;
+  if (cache[di][gi] == 0) {
+    int r = 0;
+    if (D == 128) r = G == 1 ? resident_blocks_of<128, 1>() : G == 2 ? resident_blocks_of<128, 2>()
+                    : G == 4 ? resident_blocks_of<128, 4>() : resident_blocks_of<128, 8>();
+    else r = G == 1 ? resident_blocks_of<64, 1>() : G == 2 ? resident_blocks_of<64, 2>()
+             : G == 4 ? resident_blocks_of<64, 4>() : resident_blocks_of<64, 8>();
+    if (r <= 0) { cudaGetLastError(); return 148 * 7; }
+    cache[di][gi] = r;
+  }
+  return cache[di][gi];
+}
+
+// Splits per (sequence, KV head): the grid should be a whole number of waves of resident blocks, each
+// split at most kChunkCap rows (its scores live in shared memory) and not much shorter than 128 rows.
+int pick_splits(int B, int Tmax, int Hq, int Hkv, int D, const cowa_params_t* p) {
   const int hg = p->hkv_global > 0 ? p->hkv_global : Hkv;
   const int vmax = max_visible(Tmax, hg, p);
-  // enough blocks to fill 148 SMs several times over, and splits short enough for shared memory
-  int by_fill = (148 * 16 + B * Hkv - 1) / (B * Hkv);
-  int by_cap = (vmax + (kChunkCap - 16) - 1) / (kChunkCap - 16);
-  int by_len = (vmax + 127) / 128;  // no point in splits shorter than 128 rows
-  int s = by_fill < by_len ? by_fill : by_len;
+  const int heads = B * Hkv;
+  const int by_cap = (vmax + (kChunkCap - 16) - 1) / (kChunkCap - 16);
+  const int by_len = (vmax + 127) / 128;
+  const int slots = resident_blocks(D, Hq / Hkv);
+  int s = by_cap;
+  for (int waves = 1; waves <= 64; ++waves) {
+    s = (int)(((long long)waves * slots) / heads);
+    if (s >= by_cap && s >= 1) break;
+  }
+  if (s > by_len) s = by_len;
   if (s < by_cap) s = by_cap;
   return s < 1 ? 1 : s;
 }
@@ -331,7 +423,7 @@ int decode_validate(const void* q, const void* kc, const void* vc, const int32_t
   if (G != 1 && G != 2 && G != 4 && G != 8) return COWA_ERR_UNSUPPORTED;
   if (B > 65535 || Hkv > 65535) return COWA_ERR_UNSUPPORTED;
   if (!aligned16(q) || !aligned16(kc) || !aligned16(vc) || !aligned16(o)) return COWA_ERR_MISALIGNED;
-  *S = pick_splits(B, Tmax, Hkv, p);
+  *S = pick_splits(B, Tmax, Hq, Hkv, D, p);
   return COWA_OK;
 }
 
@@ -364,7 +456,7 @@ int decode_launch(const void* q, const void* kc, const void* vc, const int32_t* 
     cowa_decode_combine_kernel<128><<<B * Hq, 128, 0, st>>>(a.ws_o, a.ws_m, a.ws_l,
                                                             static_cast<__nv_bfloat16*>(o), lse, S);
   else
-    cowa_decode_combine_kernel<64><<<B * Hq, 64, 0, st>>>(a.ws_o, a.ws_m, a.ws_l,
+    cowa_decode_combine_kernel<64><<<B * Hq, 128, 0, st>>>(a.ws_o, a.ws_m, a.ws_l,
                                                           static_cast<__nv_bfloat16*>(o), lse, S);
   e = cudaGetLastError();
   if (e != cudaSuccess) return record_cuda_error(e);
@@ -376,8 +468,8 @@ int decode_launch(const void* q, const void* kc, const void* vc, const int32_t* 
 extern "C" {
 
 size_t cowa_decode_workspace_bytes(int B, int Tmax, int Hq, int Hkv, int D, const cowa_params_t* p) {
-  if (!p || B <= 0 || Tmax <= 0 || Hq <= 0 || Hkv <= 0 || D <= 0) return 0;
-  return cowa::decode_ws_bytes(B, Hq, D, pick_splits(B, Tmax, Hkv, p));
+  if (!p || B <= 0 || Tmax <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || (D != 64 && D != 128)) return 0;
+  return cowa::decode_ws_bytes(B, Hq, D, pick_splits(B, Tmax, Hq, Hkv, D, p));
 }
 
 int cowa_decode(const void* q, const void* kcache, const void* vcache, const int32_t* lens, void* o,
