@@ -1,16 +1,19 @@
 // CoWindow Attention forward (Algorithm 1) for sm_100a.
 //
-// One thread block = one (batch, QO head, 128-row QO tile).  The block walks the tile's visited
-// KV tiles J_h(i) (analytic scheduler, descending order), and for each:
-//   TMA loads K / V tiles (128B-swizzled) -> tcgen05.mma S = Q K^T into TMEM -> each of the 128
-//   threads owns one row: tcgen05.ld, (boundary tiles only) window/causal mask from a per-row
-//   bit mask, online softmax in base 2 with the scale folded in, P written back to TMEM as
-//   bf16 over S's columns -> tcgen05.mma O += P V with P as the TMEM operand.
+// One thread block = one (batch, QO head, 128-row QO tile); it walks the tile's visited KV tiles
+// J_h(i) (analytic scheduler, descending order) in steps of 64 keys.  Five warps:
+//   warps 0-3  softmax: one query row per thread.  tcgen05.ld of S, (boundary tiles only) the
+//              window/causal mask from a per-row bit mask, online softmax in base 2 with the
+//              scale folded in, P written back to TMEM as bf16 over S's columns.
+//   warp 4     control (one lane): TMA loads of K and V (128B swizzle, two buffers each) and all
+//              tcgen05.mma issue: S = Q K^T into one of two TMEM buffers, O += P V with P as the
+//              TMEM operand.  S of step t+1 is issued before the softmax of step t starts, so the
+//              softmax threads never wait for the tensor pipe in steady state.
 // The running max is only advanced when the row max grows by more than 2^8 (the accumulator is
 // rescaled in TMEM only then); the final normalisation uses the same reference max, so the
 // result is the exact softmax.  Two blocks fit per SM (96 KB shared memory, 256 TMEM columns
-// each), which overlaps one block's softmax with the other's MMAs.  The 4 QO heads of a GQA
-// group at the same tile are adjacent in launch order and share K/V through L2.
+// each).  The QO heads of a GQA group at the same tile are adjacent in launch order and share
+// K/V through L2.
 #include <cuda_bf16.h>
 
 #include "cowa_common.h"
@@ -21,7 +24,8 @@ using namespace cowa_ptx;
 
 namespace {
 
-constexpr int BQ = 128, BK = 128;
+constexpr int BQ = 128, BK = 64;
+constexpr int kFwdThreads = 160;
 
 struct FwdArgs {
   float* lse;
@@ -40,33 +44,39 @@ __device__ __forceinline__ uint32_t interval_bits(int a, int b, int base) {
 
 template <int D>
 struct FwdSmem {
-  static constexpr int kTile = 128 * D * 2;  // bytes of one 128-row tile
-  static constexpr int kQ = 0, kK = kTile, kV = 2 * kTile, kBar = 3 * kTile;
-  static constexpr int kBytes = 3 * kTile + 64 + 1024;  // + barriers + alignment slack
+  static constexpr int kQ = BQ * D * 2;   // Q tile (later the O staging tile)
+  static constexpr int kKV = BK * D * 2;  // one K or V step tile
+  static constexpr int oQ = 0, oK = kQ, oV = kQ + 2 * kKV, oBar = kQ + 4 * kKV;
+  static constexpr int kBytes = oBar + 128 + 1024;  // + barriers + alignment slack
 };
 
 template <int D>
-__global__ void __launch_bounds__(128, 2)
+__global__ void __launch_bounds__(kFwdThreads, 2)
 cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
                 const __grid_constant__ FwdArgs a) {
+  using SM = FwdSmem<D>;
   constexpr int NSLAB = D / 64;          // 64-element (128-byte) slabs along D
-  constexpr int SLAB = 128 * 128;        // bytes of one slab: 128 rows x 128 B
-  constexpr uint32_t TMEM_COLS = 256;    // S/P: [0,128), O: [128, 128+D)
+  constexpr int SLAB_Q = BQ * 128;       // bytes of one slab of a 128-row tile
+  constexpr int SLAB_K = BK * 128;       // ... of a 64-row tile
+  constexpr uint32_t TMEM_COLS = 256;    // S/P buffers: [0,64), [64,128); O: [128, 128+D)
+  constexpr uint32_t cO = 128;
   constexpr uint32_t IDESC_S = idesc_bf16(128, BK, 0, 0);
   constexpr uint32_t IDESC_O = idesc_bf16(128, D, 0, 1);
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* sQ = smem + FwdSmem<D>::kQ;
-  uint8_t* sK = smem + FwdSmem<D>::kK;
-  uint8_t* sV = smem + FwdSmem<D>::kV;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + FwdSmem<D>::kBar);
+  uint8_t* sQ = smem + SM::oQ;
+  uint8_t* sK = smem + SM::oK;  // [2][kKV]
+  uint8_t* sV = smem + SM::oV;  // [2][kKV]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::oBar);
   uint64_t* bar_q = bars + 0;
-  uint64_t* bar_k = bars + 1;
-  uint64_t* bar_v = bars + 2;
-  uint64_t* bar_mma = bars + 3;
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 4);
+  uint64_t* bar_k = bars + 1;   // [2] K step tile landed
+  uint64_t* bar_v = bars + 3;   // [2] V step tile landed
+  uint64_t* bar_s = bars + 5;   // [2] S of a step is in TMEM buffer b
+  uint64_t* bar_p = bars + 7;   // [2] count 128: P written over S
+  uint64_t* bar_pv = bars + 9;  //     O += P V of a step has completed
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 10);
 
   const int tid = threadIdx.x, warp = tid >> 5;
 
@@ -83,14 +93,17 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const CowaWin w = a.wins.w[hk];
   CowaRange rg[3];
   cowa_fwd_ranges(w, q0, q1, off, a.Nk, BK, rg);
-  const int ntiles = cowa_range_len(rg[0]) + cowa_range_len(rg[1]) + cowa_range_len(rg[2]);
+  const int nt = cowa_range_len(rg[0]) + cowa_range_len(rg[1]) + cowa_range_len(rg[2]);
   const int bhq = b * a.Hq + h, bhk = b * a.Hkv + hk;
 
   // ---- set-up ----
   if (tid == 0) {
-    mbar_init(bar_q, 1); mbar_init(bar_k, 1); mbar_init(bar_v, 1); mbar_init(bar_mma, 1);
+    mbar_init(bar_q, 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(bar_k + s, 1); mbar_init(bar_v + s, 1); mbar_init(bar_s + s, 1); mbar_init(bar_p + s, 128);
+    }
+    mbar_init(bar_pv, 1);
     fence_mbar_init();
-    prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV); prefetch_tmap(&tmO);
   }
   if (warp == 0) {
     __syncwarp();
@@ -101,194 +114,199 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
-  const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);  // this warp's 32 lanes
-  const uint32_t t_S = t_lane, t_O = t_lane + 128;
 
-  bool ok = true;  // false once a bounded wait ran out
-  uint32_t ph_k = 0, ph_v = 0, ph_mma = 0;
+  bool ok = true;  // false once a bounded wait ran out; every role then falls through to the teardown
 
-  if (tid == 0 && ntiles > 0) {
-    const int j0 = cowa_fwd_tile_at(rg, 0);
-    mbar_expect_tx(bar_q, FwdSmem<D>::kTile);
-    for (int s = 0; s < NSLAB; ++s) tma_load_3d(sQ + s * SLAB, &tmQ, bar_q, s * 64, q0, bhq);
-    mbar_expect_tx(bar_k, FwdSmem<D>::kTile);
-    for (int s = 0; s < NSLAB; ++s) tma_load_3d(sK + s * SLAB, &tmK, bar_k, s * 64, j0 * BK, bhk);
-    mbar_expect_tx(bar_v, FwdSmem<D>::kTile);
-    for (int s = 0; s < NSLAB; ++s) tma_load_3d(sV + s * SLAB, &tmV, bar_v, s * 64, j0 * BK, bhk);
-  }
-
-  // ---- per-row state ----
-  const int row = q0 + tid;
-  const bool row_valid = row < a.Nq;
-  const int rowpos = row + off;  // position of this query on the key axis
-  float m_ref = -INFINITY, l_sum = 0.f;
-
-  for (int t = 0; t < ntiles; ++t) {
-    const int j = cowa_fwd_tile_at(rg, t);
-    const int k0 = j * BK;
-    const bool full = cowa_tile_full(w, q0, BQ, k0, BK, off, a.Nq, a.Nk);
-
-    // Thread 0 never leaves the loop on its own: a failed wait only clears `ok`, and every
-    // thread leaves together at the block-wide vote below.
-    if (tid == 0) {
-      if (t == 0) ok = ok && mbar_wait(bar_q, 0, a.status);
-      ok = ok && mbar_wait(bar_k, ph_k, a.status);
-      ph_k ^= 1;
-      if (ok) {
-        tc_fence_after();
+  if (warp == 4) {
+    // ======================= control: TMA loads and MMA issue (one lane) =======================
+    if (tid == 128 && nt > 0) {
+      prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV);
+      auto load_k = [&](int t) {
+        const int j = cowa_fwd_tile_at(rg, t);
+        uint8_t* dst = sK + (t & 1) * SM::kKV;
+        mbar_expect_tx(bar_k + (t & 1), SM::kKV);
+        for (int s = 0; s < NSLAB; ++s) tma_load_3d(dst + s * SLAB_K, &tmK, bar_k + (t & 1), s * 64, j * BK, bhk);
+      };
+      auto load_v = [&](int t) {
+        const int j = cowa_fwd_tile_at(rg, t);
+        uint8_t* dst = sV + (t & 1) * SM::kKV;
+        mbar_expect_tx(bar_v + (t & 1), SM::kKV);
+        for (int s = 0; s < NSLAB; ++s) tma_load_3d(dst + s * SLAB_K, &tmV, bar_v + (t & 1), s * 64, j * BK, bhk);
+      };
+      const uint64_t dQ = smem_desc_sw128(smem_u32(sQ), 16, 1024);
+      auto issue_s = [&](int t) {  // S(t) = Q K(t)^T into buffer t & 1
+        const uint64_t dK = smem_desc_sw128(smem_u32(sK + (t & 1) * SM::kKV), 16, 1024);
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t o = (kk / 4) * SLAB + (kk % 4) * 32;
-          mma_ss(tmem_base, smem_desc_sw128(smem_u32(sQ) + o, 16, 1024), smem_desc_sw128(smem_u32(sK) + o, 16, 1024),
-                 IDESC_S, kk > 0);
+        for (int kk = 0; kk < D / 16; ++kk)
+          mma_ss(tmem_base + (t & 1) * 64, dQ + (((kk / 4) * SLAB_Q + (kk % 4) * 32) >> 4),
+                 dK + (((kk / 4) * SLAB_K + (kk % 4) * 32) >> 4), IDESC_S, kk > 0);
+        mma_commit(bar_s + (t & 1));
+      };
+      mbar_expect_tx(bar_q, SM::kQ);
+      for (int s = 0; s < NSLAB; ++s) tma_load_3d(sQ + s * SLAB_Q, &tmQ, bar_q, s * 64, q0, bhq);
+      load_k(0);
+      if (nt > 1) load_k(1);
+      load_v(0);
+      ok = mbar_wait(bar_q, 0, a.status) && mbar_wait(bar_k, 0, a.status);
+      if (ok) { tc_fence_after(); issue_s(0); }
+      for (int t = 0; t < nt && ok; ++t) {
+        const int b_ = t & 1;
+        const uint32_t par = (t >> 1) & 1;
+        if (t + 1 < nt) {  // S(t+1): its buffer last held P(t-1), whose product was issued before this one
+          ok = mbar_wait(bar_k + (b_ ^ 1), ((t + 1) >> 1) & 1, a.status);
+          if (!ok) break;
+          tc_fence_after();
+          issue_s(t + 1);
+        }
+        if (t + 2 < nt) {  // K(t+2) over K(t), once S(t) has been computed
+          ok = mbar_wait(bar_s + b_, par, a.status);
+          if (!ok) break;
+          load_k(t + 2);
+        }
+        if (t + 1 < nt) {  // V(t+1) over V(t-1), once O += P V of step t-1 has completed
+          if (t >= 1) ok = mbar_wait(bar_pv, (t - 1) & 1, a.status);
+          if (!ok) break;
+          load_v(t + 1);
+        }
+        ok = mbar_wait(bar_p + b_, par, a.status) && mbar_wait(bar_v + b_, par, a.status);
+        if (!ok) break;
+        tc_fence_after();
+        const uint64_t dV = smem_desc_sw128(smem_u32(sV + b_ * SM::kKV), SLAB_K, 1024);
+#pragma unroll
+        for (int kk = 0; kk < BK / 16; ++kk)
+          mma_ts(tmem_base + cO, tmem_base + b_ * 64 + kk * 8, dV + ((kk * 2048) >> 4), IDESC_O,
+                 (t > 0 || kk > 0) ? 1u : 0u);
+        mma_commit(bar_pv);
+      }
+    }
+  } else {
+    // ======================= softmax: one query row per thread =======================
+    const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);  // this warp's 32 lanes
+    const uint32_t t_O = t_lane + cO;
+    const int row = q0 + tid;
+    const bool row_valid = row < a.Nq;
+    const int rowpos = row + off;  // position of this query on the key axis
+    float m_ref = -INFINITY, l_sum = 0.f;
+    const float2 sc2 = make_float2(a.scale_log2, a.scale_log2);
+
+    for (int t = 0; t < nt && ok; ++t) {
+      const int b_ = t & 1;
+      const int j = cowa_fwd_tile_at(rg, t);
+      const int k0 = j * BK;
+      const bool full = cowa_tile_full(w, q0, BQ, k0, BK, off, a.Nq, a.Nk);
+      const uint32_t t_S = t_lane + b_ * 64;
+
+      ok = mbar_wait(bar_s + b_, (t >> 1) & 1, a.status);
+      if (!ok) break;
+      tc_fence_after();
+      uint32_t sr[2][32];
+      tmem_ld32(t_S, sr[0]);
+      tmem_ld32(t_S + 32, sr[1]);
+      tmem_wait_ld();
+
+      if (!full) {
+        const int kend = min(rowpos, a.Nk - 1);  // last causal key of this row
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          const int base = k0 + c * 32;
+          uint32_t mk = interval_bits(rowpos - w.n + 1, kend, base) | interval_bits(0, min(w.s - 1, kend), base);
+          if (w.l > 0) mk |= interval_bits(rowpos - (w.n + w.g + w.l) + 1, min(rowpos - (w.n + w.g), kend), base);
+          if (!row_valid) mk = 0u;
+#pragma unroll
+          for (int e = 0; e < 32; ++e)
+            if (!((mk >> e) & 1u)) sr[c][e] = 0xFF800000u;  // -inf
         }
       }
-      mma_commit(bar_mma);
+      // row max: four independent chains of 3-input max
+      float mxa[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+      for (int c = 0; c < 2; ++c)
+#pragma unroll
+        for (int e = 0; e < 32; e += 2)
+          mxa[(e >> 1) & 3] = max3(mxa[(e >> 1) & 3], __uint_as_float(sr[c][e]), __uint_as_float(sr[c][e + 1]));
+      const float mx = fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3])) * a.scale_log2;
+      float m_new = m_ref;
+      if (mx > m_ref + 8.f) m_new = mx;
+      const float alpha = (m_new == m_ref) ? 1.f : ex2(m_ref - m_new);
+      const float sub = (m_new == -INFINITY) ? 0.f : m_new;
+      m_ref = m_new;
+
+      // p = 2^(s * scale - m): packed fp32 pairs for the multiply-add and the row sum
+      const float2 nsub2 = make_float2(-sub, -sub);
+      float2 rsa[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+      uint32_t pk[32];
+#pragma unroll
+      for (int c = 0; c < 2; ++c)
+#pragma unroll
+        for (int e = 0; e < 32; e += 2) {
+          const float2 x = fma2(make_float2(__uint_as_float(sr[c][e]), __uint_as_float(sr[c][e + 1])), sc2, nsub2);
+          const float2 pp = make_float2(ex2(x.x), ex2(x.y));
+          rsa[(e >> 1) & 3] = add2(rsa[(e >> 1) & 3], pp);
+          pk[c * 16 + e / 2] = pack_bf16(pp.x, pp.y);
+        }
+      const float2 rs2 = add2(add2(rsa[0], rsa[1]), add2(rsa[2], rsa[3]));
+      l_sum = l_sum * alpha + (rs2.x + rs2.y);
+
+      // Every step waits for the product of the step before (normally long finished): the accumulator
+      // may then be rescaled safely, and no thread ever falls two phases behind on this barrier, which
+      // its parity wait could not tell apart.
+      if (t > 0) {
+        ok = mbar_wait(bar_pv, (t - 1) & 1, a.status);
+        if (!ok) break;
+        tc_fence_after();
+      }
+      // rescale the accumulator when some row of this warp moved its reference max
+      if (t > 0 && __any_sync(0xFFFFFFFFu, alpha != 1.f)) {
+        const float2 al2 = make_float2(alpha, alpha);
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t ov[32];
+          tmem_ld32(t_O + c * 32, ov);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            const float2 y = mul2(make_float2(__uint_as_float(ov[e]), __uint_as_float(ov[e + 1])), al2);
+            ov[e] = __float_as_uint(y.x); ov[e + 1] = __float_as_uint(y.y);
+          }
+          tmem_st32(t_O + c * 32, ov);
+        }
+      }
+      tmem_st32(t_S, pk);  // P over the first 32 columns of this S buffer
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar_p + b_);
     }
-    __syncwarp();
-    ok = mbar_wait(bar_mma, ph_mma, a.status) && ok;
-    ph_mma ^= 1;
-    ok = __syncthreads_and(ok);
-    if (!ok) break;
-    tc_fence_after();
 
-    if (tid == 0) {  // S(t) is in TMEM, PV(t-1) is complete: both operand buffers are free again
-      if (t + 1 < ntiles) {
-        const int jn = cowa_fwd_tile_at(rg, t + 1);
-        mbar_expect_tx(bar_k, FwdSmem<D>::kTile);
-        for (int s = 0; s < NSLAB; ++s) tma_load_3d(sK + s * SLAB, &tmK, bar_k, s * 64, jn * BK, bhk);
-      }
-      if (t >= 1) {
-        mbar_expect_tx(bar_v, FwdSmem<D>::kTile);
-        for (int s = 0; s < NSLAB; ++s) tma_load_3d(sV + s * SLAB, &tmV, bar_v, s * 64, k0, bhk);
-      }
-    }
-    __syncwarp();
-
-    // ---- this thread's row of S ----
-    uint32_t sr[4][32];
-#pragma unroll
-    for (int c = 0; c < 4; ++c) tmem_ld32(t_S + c * 32, sr[c]);
-    tmem_wait_ld();
-
-    uint32_t mask[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};
-    if (!full) {
-      const int kend = min(rowpos, a.Nk - 1);  // last causal key of this row
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const int base = k0 + c * 32;
-        uint32_t mk = interval_bits(rowpos - w.n + 1, kend, base) | interval_bits(0, min(w.s - 1, kend), base);
-        if (w.l > 0) mk |= interval_bits(rowpos - (w.n + w.g + w.l) + 1, min(rowpos - (w.n + w.g), kend), base);
-        mask[c] = row_valid ? mk : 0u;
-      }
-    }
-    // row max: four independent chains of 3-input max
-    float mxa[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      if (!full) {
-#pragma unroll
-        for (int e = 0; e < 32; ++e)
-          if (!((mask[c] >> e) & 1u)) sr[c][e] = 0xFF800000u;  // -inf
-      }
-#pragma unroll
-      for (int e = 0; e < 32; e += 2)
-        mxa[(e >> 1) & 3] = max3(mxa[(e >> 1) & 3], __uint_as_float(sr[c][e]), __uint_as_float(sr[c][e + 1]));
-    }
-    const float mx = fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3])) * a.scale_log2;
-    float m_new = m_ref;
-    if (mx > m_ref + 8.f) m_new = mx;
-    const float alpha = (m_new == m_ref) ? 1.f : ex2(m_ref - m_new);
-    const float sub = (m_new == -INFINITY) ? 0.f : m_new;
-    m_ref = m_new;
-
-    // p = 2^(s * scale - m): packed fp32 pairs for the multiply-add and the row sum
-    const float2 sc2 = make_float2(a.scale_log2, a.scale_log2), nsub2 = make_float2(-sub, -sub);
-    float2 rsa[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-    uint32_t pk[64];
-#pragma unroll
-    for (int c = 0; c < 4; ++c)
-#pragma unroll
-      for (int e = 0; e < 32; e += 2) {
-        const float2 x = fma2(make_float2(__uint_as_float(sr[c][e]), __uint_as_float(sr[c][e + 1])), sc2, nsub2);
-        const float2 pp = make_float2(ex2(x.x), ex2(x.y));
-        rsa[(e >> 1) & 3] = add2(rsa[(e >> 1) & 3], pp);
-        pk[c * 16 + e / 2] = pack_bf16(pp.x, pp.y);
-      }
-    const float2 rs2 = add2(add2(rsa[0], rsa[1]), add2(rsa[2], rsa[3]));
-    l_sum = l_sum * alpha + (rs2.x + rs2.y);
-
-    // P over S's first 64 columns
-#pragma unroll
-    for (int c = 0; c < 4; ++c) tmem_st16(t_S + c * 16, &pk[c * 16]);
-
-    // rescale the accumulator when some row of this warp moved its reference max
-    if (t > 0 && __any_sync(0xFFFFFFFFu, alpha != 1.f)) {
+    // ---- epilogue: O / l, LSE ----
+    if (nt > 0) ok = mbar_wait(bar_pv, (nt - 1) & 1, a.status) && ok;
+    if (ok && nt > 0) {
+      tc_fence_after();
+      const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
 #pragma unroll
       for (int c = 0; c < D / 32; ++c) {
         uint32_t ov[32];
         tmem_ld32(t_O + c * 32, ov);
         tmem_wait_ld();
+        // 32 columns = 4 chunks of 8 elements (16 B); slab = (c*32)/64, chunk index within slab
 #pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-          const float2 y = mul2(make_float2(__uint_as_float(ov[e]), __uint_as_float(ov[e + 1])), make_float2(alpha, alpha));
-          ov[e] = __float_as_uint(y.x); ov[e + 1] = __float_as_uint(y.y);
-        }
-        tmem_st32(t_O + c * 32, ov);
-      }
-    }
-    tmem_wait_st();
-    tc_fence_before();
-    __syncthreads();
-
-    if (tid == 0) {
-      ok = ok && mbar_wait(bar_v, ph_v, a.status);
-      ph_v ^= 1;
-      if (ok) {
-        tc_fence_after();
-#pragma unroll
-        for (int kk = 0; kk < BK / 16; ++kk) {
-          mma_ts(tmem_base + 128, tmem_base + kk * 8, smem_desc_sw128(smem_u32(sV) + kk * 2048, SLAB, 1024), IDESC_O,
-                 (t > 0 || kk > 0) ? 1u : 0u);
+        for (int q = 0; q < 4; ++q) {
+          uint4 v;
+          v.x = pack_bf16(__uint_as_float(ov[q * 8 + 0]) * inv, __uint_as_float(ov[q * 8 + 1]) * inv);
+          v.y = pack_bf16(__uint_as_float(ov[q * 8 + 2]) * inv, __uint_as_float(ov[q * 8 + 3]) * inv);
+          v.z = pack_bf16(__uint_as_float(ov[q * 8 + 4]) * inv, __uint_as_float(ov[q * 8 + 5]) * inv);
+          v.w = pack_bf16(__uint_as_float(ov[q * 8 + 6]) * inv, __uint_as_float(ov[q * 8 + 7]) * inv);
+          const int d0 = c * 32 + q * 8;
+          const int slab = d0 / 64, chunk = (d0 % 64) / 8;
+          *reinterpret_cast<uint4*>(sQ + slab * SLAB_Q + tid * 128 + ((chunk ^ (tid & 7)) << 4)) = v;
         }
       }
-      if (t == ntiles - 1) mma_commit(bar_mma);
+      if (row_valid)
+        a.lse[(size_t)bhq * a.Nq + row] = 0.6931471805599453f * (m_ref + log2f(l_sum));
+      fence_proxy_async_smem();
     }
-    __syncwarp();
-  }
-
-  // ---- epilogue: O / l, LSE ----
-  if (ntiles > 0) {
-    ok = mbar_wait(bar_mma, ph_mma, a.status) && ok;
-    ok = __syncthreads_and(ok);
-  }
-  if (ok && ntiles > 0) {
-    tc_fence_after();
-    const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
-#pragma unroll
-    for (int c = 0; c < D / 32; ++c) {
-      uint32_t ov[32];
-      tmem_ld32(t_O + c * 32, ov);
-      tmem_wait_ld();
-      // 32 columns = 4 chunks of 8 elements (16 B); slab = (c*32)/64, chunk index within slab
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        uint4 v;
-        v.x = pack_bf16(__uint_as_float(ov[q * 8 + 0]) * inv, __uint_as_float(ov[q * 8 + 1]) * inv);
-        v.y = pack_bf16(__uint_as_float(ov[q * 8 + 2]) * inv, __uint_as_float(ov[q * 8 + 3]) * inv);
-        v.z = pack_bf16(__uint_as_float(ov[q * 8 + 4]) * inv, __uint_as_float(ov[q * 8 + 5]) * inv);
-        v.w = pack_bf16(__uint_as_float(ov[q * 8 + 6]) * inv, __uint_as_float(ov[q * 8 + 7]) * inv);
-        const int d0 = c * 32 + q * 8;
-        const int slab = d0 / 64, chunk = (d0 % 64) / 8;
-        *reinterpret_cast<uint4*>(sQ + slab * SLAB + tid * 128 + ((chunk ^ (tid & 7)) << 4)) = v;
-      }
-    }
-    if (row_valid)
-      a.lse[(size_t)bhq * a.Nq + row] = 0.6931471805599453f * (m_ref + log2f(l_sum));
-    fence_proxy_async_smem();
-    __syncthreads();
-    if (tid == 0) {
-      for (int s = 0; s < NSLAB; ++s) tma_store_3d(&tmO, sQ + s * SLAB, s * 64, q0, bhq);
+    asm volatile("bar.sync 1, 128;" ::: "memory");  // the four softmax warps
+    if (tid == 0 && ok && nt > 0) {
+      for (int s = 0; s < NSLAB; ++s) tma_store_3d(&tmO, sQ + s * SLAB_Q, s * 64, q0, bhq);
       tma_commit_group();
       tma_wait_group<0>();
     }
@@ -323,7 +341,7 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
                                      FwdSmem<D>::kBytes));
   const long long nblocks = (long long)((T + BQ - 1) / BQ) * B * Hq;
   if (nblocks > 0x7FFFFFFFll) return COWA_ERR_UNSUPPORTED;
-  cowa_fwd_kernel<D><<<(unsigned)nblocks, 128, FwdSmem<D>::kBytes, st>>>(mq, mk, mv, mo, a);
+  cowa_fwd_kernel<D><<<(unsigned)nblocks, kFwdThreads, FwdSmem<D>::kBytes, st>>>(mq, mk, mv, mo, a);
   COWA_CUDA_TRY(cudaGetLastError());
   return COWA_OK;
 }
