@@ -202,6 +202,63 @@ def test_bwd_8k_config_sampled():
         check_grad(f"dv[{b},{hk},{tile}]", dv[b, hk, cols].float().cpu().numpy(), dv_r)
 
 
+# ------------------------------------------------------------------ full-size configurations, sampled
+
+def _full_size_sampled(name, q_tiles, kv_samples):
+    """Runs forward + backward at a benchmark configuration in the launch configuration bench.py
+    times, and compares sampled outputs with the oracle: O/LSE/dQ on whole 128-row query tiles,
+    dK/dV on whole 128-row KV tiles (each needs every query row that sees the tile)."""
+    c = cowa_inputs.CONFIGS[name]
+    B, T, Hq, Hkv, D = c["B"], c["T"], c["Hq"], c["Hkv"], c["D"]
+    q, k, v, d_o = cowa_inputs.make_train_inputs(c["index"], B, T, Hq, Hkv, D, device=DEV)
+    scale = cowa_inputs.softmax_scale(D)
+    params = cowa.make_params(sink=c["sink"], local=c["local"], softmax_scale=scale)
+    o, lse = run_fwd(q, k, v, params)
+    dq, dk, dv = (torch.empty_like(x) for x in (q, k, v))
+    ws_b = torch.empty(cowa.cowa_bwd_workspace_bytes(B, T, Hq, Hkv, D, params), dtype=torch.uint8, device=DEV)
+    cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, params, ws_b)
+    torch.cuda.synchronize()
+    cowa.cowa_check_device_status()
+    del ws_b
+    ws = orc.default_windows(T, Hkv, c["sink"], c["local"])
+    f = cowa_inputs.to_f64
+    G = Hq // Hkv
+    cache = {}
+
+    def head_inputs(h):  # float64 copies of one QO head and its KV head, shaped like a 1-head problem
+        hk = h // G
+        if hk not in cache:
+            cache.clear()
+            cache[hk] = (f(k[0, hk:hk + 1]), f(v[0, hk:hk + 1]))
+        return f(q[0, h:h + 1]), cache[hk][0], cache[hk][1], f(d_o[0, h:h + 1]), [ws[hk]]
+
+    for h, tile in q_tiles:
+        rows = np.arange(tile * 128, tile * 128 + 128)
+        qh, kh, vh, doh, w1 = head_inputs(h)
+        o_ref, lse_ref = orc.forward_rows(qh, kh, vh, w1, scale, 0, rows)
+        check(f"{name} lse[h{h},tile{tile}]", lse[0, h, rows].cpu().numpy(), lse_ref, TOL_LSE, TOL_LSE)
+        check(f"{name} o[h{h},tile{tile}]", o[0, h, rows].float().cpu().numpy(), o_ref)
+        dq_ref = orc.backward_dq_rows(qh, kh, vh, doh, w1, scale, 0, rows)
+        check_grad(f"{name} dq[h{h},tile{tile}]", dq[0, h, rows].float().cpu().numpy(), dq_ref)
+    for hk, tile in kv_samples:
+        cols = np.arange(tile * 128, tile * 128 + 128)
+        qg, dog = f(q[0, hk * G:(hk + 1) * G]), f(d_o[0, hk * G:(hk + 1) * G])
+        dk_r, dv_r = orc.backward_dkdv_cols(qg, f(k[0, hk:hk + 1]), f(v[0, hk:hk + 1]), dog, [ws[hk]], scale, 0, cols)
+        check_grad(f"{name} dk[hk{hk},tile{tile}]", dk[0, hk, cols].float().cpu().numpy(), dk_r)
+        check_grad(f"{name} dv[hk{hk},tile{tile}]", dv[0, hk, cols].float().cpu().numpy(), dv_r)
+
+
+def test_32k_config_sampled():
+    # query tiles: first, last, and tiles whose rows straddle a band edge of their head
+    _full_size_sampled("32k", q_tiles=[(0, 0), (3, 255), (9, 17), (14, 100), (31, 255), (20, 46)],
+                       kv_samples=[(0, 0), (2, 77), (7, 255)])
+
+
+def test_128k_config_sampled():
+    _full_size_sampled("128k", q_tiles=[(0, 1023), (5, 33), (13, 500), (31, 1023), (18, 157)],
+                       kv_samples=[(6, 901)])
+
+
 # ------------------------------------------------------------------ decode
 
 def run_decode(q, kc, vc, lens, params):
