@@ -259,12 +259,19 @@ def run_cuda(args):
         have_bwd = False
     torch.cuda.synchronize()
 
-    def step(params, ev=None):
+    main_evs = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
+    for pair in main_evs:
+        for e_ in pair:
+            e_.record()  # creates the underlying CUDA event
+
+    def step(params, ev=None, main_ev=None):
         if ev: ev[0].record()
         cowa.cowa_fwd(q, k, v, o, lse, params)
         if ev: ev[1].record()
         if have_bwd:
+            if main_ev: cowa.cowa_bwd_set_profile_events(main_ev[0], main_ev[1])
             cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, params, ws_bwd)
+            if main_ev: cowa.cowa_bwd_set_profile_events(None, None)
         if ev: ev[2].record()
         cowa.cowa_decode(qd, kc, vc, lens, od, lsed, p_dec, ws_dec)
         if ev: ev[3].record()
@@ -280,7 +287,7 @@ def run_cuda(args):
         sampler.start()
     barrier(world)
     for s in range(args.steps):
-        step(p_train, evs[s])
+        step(p_train, evs[s], main_evs[s])
     barrier(world)
     clocks = sampler.stop() if rank == 0 else None
     cowa.cowa_check_device_status()
@@ -291,6 +298,10 @@ def run_cuda(args):
     total_ms = evs[0][0].elapsed_time(evs[-1][3]) / args.steps
     fwd_ms, bwd_ms, dec_ms, total_ms = (max_over_ranks(x, world) for x in (fwd_ms, bwd_ms, dec_ms, total_ms))
 
+    # main backward kernel alone (the call also enqueues a memset, the preprocess and the dQ conversion)
+    bwd_main_ms = None
+    if have_bwd:
+        bwd_main_ms = max_over_ranks(sum(e[0].elapsed_time(e[1]) for e in main_evs) / args.steps, world)
     train_flops = fwd_flops + (bwd_flops if have_bwd else 0.0)
     train_ms = fwd_ms + (bwd_ms if have_bwd else 0.0)
     value = world * train_flops / (train_ms * 1e-3) / 1e12
@@ -367,14 +378,19 @@ def run_cuda(args):
 
     # ---- roofline of the dominant kernel ----
     if have_bwd and bwd_ms >= fwd_ms:
-        dom, dom_flops, dom_ms = "cowa_bwd main kernel", bwd_flops, bwd_ms
+        dom, dom_flops, dom_ms = "cowa_bwd_kernel<128>", bwd_flops, bwd_main_ms
     else:
         dom, dom_flops, dom_ms = "cowa_fwd_kernel<128>", fwd_flops, fwd_ms
     peak_tf = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
     achieved = dom_flops / dom_ms / 1e9
+    # DRAM bytes per launch of the dominant kernel at the 128K workload, from the one-pass ncu capture
+    # summarised in profiles/launch_list_bench_128k.md (dram__bytes_read.sum + dram__bytes_write.sum).
+    traffic_128k = {"cowa_bwd_kernel<128>": 12.876e9 + 6.633e9, "cowa_fwd_kernel<128>": 10.145e9 + 1.054e9}
     roofline = {"kernel": dom, "bound": "tensor", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s",
                 "frac": achieved / peak_tf, "peak_source": f"{peak_src} bf16 sustained (kernel timed inside a long step)",
-                "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "traffic": None}
+                "frac_of_burst_peak": achieved / peaks["bf16_tflops"],
+                "traffic": traffic_128k.get(dom) if args.train_cfg == "128k" else None,
+                "traffic_unit": "bytes per launch (ncu, 128K workload)"}
     dec_gbs = dec_bytes / (dec_ms * 1e-3) / 1e9
     decode = {"us_per_step": dec_ms * 1e3, "us_per_token": dec_ms * 1e3 / cd["B"], "visible_kv_bytes": dec_bytes,
               "achieved_gbs": dec_gbs, "hbm_peak_gbs": peaks["hbm_gbs"], "frac_hbm": dec_gbs / peaks["hbm_gbs"]}
@@ -397,6 +413,7 @@ def run_cuda(args):
                    "parallelism": "independent replicas" if world > 1 else "single GPU"},
         "fwd_ms": fwd_ms, "fwd_tflops": fwd_flops / fwd_ms / 1e9,
         "bwd_ms": bwd_ms if have_bwd else None, "bwd_tflops": bwd_flops / bwd_ms / 1e9 if have_bwd else None,
+        "bwd_main_kernel_ms": bwd_main_ms,
         "visited_tiles": cnt["visited"], "causal_tiles": cnt["causal"],
         "decode": decode, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
         "gpu_launches": args.steps * (1 + (BWD_LAUNCHES if have_bwd else 0) + 2),

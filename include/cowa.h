@@ -83,6 +83,12 @@ int cowa_bwd(const void* q, const void* k, const void* v, const void* o, const f
              int B, int T, int Hq, int Hkv, int D, const cowa_params_t* p,
              void* workspace, size_t workspace_bytes, void* stream);
 
+/* Profiling hook (no counterpart in the paper).  cowa_bwd enqueues a memset, a preprocess kernel, the
+ * main kernel (Algorithm 2's loops) and a dQ conversion kernel.  After this call, every cowa_bwd issued
+ * from the same host thread records `start_event` just before and `stop_event` just after the main kernel
+ * on the call's stream (both are cudaEvent_t handles owned by the caller; NULL, NULL switches it off). */
+int cowa_bwd_set_profile_events(void* start_event, void* stop_event);
+
 /* Single-token decode over a KV cache (Sec. 2.3 "Decoding"): the forward with N_q = 1.
  *   q [B,Hq,D]; kcache,vcache [B,Hkv,Tmax,D]; lens int32 [B] on the DEVICE, lens[b] = N_k
  *   = cached tokens + 1, the current token's K/V already stored at index lens[b]-1.

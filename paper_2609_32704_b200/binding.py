@@ -56,6 +56,8 @@ def lib():
         L.cowa_decode_static.restype = i32
         L.cowa_decode_static_capacity.argtypes = []
         L.cowa_decode_static_capacity.restype = sz
+        L.cowa_bwd_set_profile_events.argtypes = [vp, vp]
+        L.cowa_bwd_set_profile_events.restype = i32
         L.cowa_bwd_workspace_bytes.argtypes = [i32] * 5 + [pp]
         L.cowa_bwd_workspace_bytes.restype = sz
         L.cowa_decode_workspace_bytes.argtypes = [i32] * 5 + [pp]
@@ -140,6 +142,13 @@ def cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, params, workspace):
     _check(lib().cowa_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(d_o), _ptr(dq), _ptr(dk),
                           _ptr(dv), B, T, Hq, Hkv, D, C.byref(params), _ptr(workspace),
                           workspace.numel() * workspace.element_size(), _stream()), "cowa_bwd")
+
+
+def cowa_bwd_set_profile_events(start_event, stop_event):
+    """torch.cuda.Event pair (already created, e.g. recorded once) to be recorded around the main
+    backward kernel of the following cowa_bwd calls; (None, None) switches the hook off."""
+    h = lambda e: C.c_void_p(0 if e is None else e.cuda_event)
+    _check(lib().cowa_bwd_set_profile_events(h(start_event), h(stop_event)), "cowa_bwd_set_profile_events")
 
 
 def cowa_decode_workspace_bytes(B, Tmax, Hq, Hkv, D, params):

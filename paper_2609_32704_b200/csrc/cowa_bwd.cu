@@ -513,6 +513,9 @@ __global__ void cowa_bwd_convert_dq_kernel(const float* __restrict__ acc, __nv_b
   *reinterpret_cast<uint4*>(dq + ((size_t)bh * T + t) * D + part * 8) = v;
 }
 
+// Optional CUDA events recorded around the main kernel of the next cowa_bwd calls on this host thread.
+thread_local cudaEvent_t g_ev_main_start = nullptr, g_ev_main_stop = nullptr;
+
 size_t ws_bytes(int B, int T, int Hq, int D) {
   const size_t Tpad = ((size_t)T + BQS - 1) / BQS * BQS;
   return (size_t)B * Hq * Tpad * ((size_t)D + 2) * sizeof(float);
@@ -560,8 +563,10 @@ int launch_bwd(const void* q, const void* k, const void* v, const void* o, const
                                      BwdSmem<D>::kBytes));
   const long long nblocks = (long long)((T + BKV - 1) / BKV) * B * Hkv;
   if (nblocks > 0x7FFFFFFFll) return COWA_ERR_UNSUPPORTED;
+  if (g_ev_main_start) COWA_CUDA_TRY(cudaEventRecord(g_ev_main_start, st));
   cowa_bwd_kernel<D><<<(unsigned)nblocks, 512, BwdSmem<D>::kBytes, st>>>(mq, mk, mv, mdo, mdk, mdv, mdq, a);
   COWA_CUDA_TRY(cudaGetLastError());
+  if (g_ev_main_stop) COWA_CUDA_TRY(cudaEventRecord(g_ev_main_stop, st));
   {
     const long long threads = BH * T * (D / 8);
     cowa_bwd_convert_dq_kernel<D><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(
@@ -574,6 +579,12 @@ int launch_bwd(const void* q, const void* k, const void* v, const void* o, const
 }  // namespace
 
 extern "C" {
+
+int cowa_bwd_set_profile_events(void* start_event, void* stop_event) {
+  g_ev_main_start = static_cast<cudaEvent_t>(start_event);
+  g_ev_main_stop = static_cast<cudaEvent_t>(stop_event);
+  return COWA_OK;
+}
 
 size_t cowa_bwd_workspace_bytes(int B, int T, int Hq, int Hkv, int D, const cowa_params_t* p) {
   (void)Hkv; (void)p;
