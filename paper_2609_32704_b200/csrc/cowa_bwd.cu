@@ -26,6 +26,7 @@
 #include <cuda_bf16.h>
 
 #include <algorithm>
+#include <type_traits>
 
 #include "cowa_common.h"
 #include "cowa_ptx.cuh"
@@ -119,7 +120,8 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   uint64_t* bar_done = bars + 13 + 2 * NST;
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 14 + 2 * NST);
 
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);  // warp-uniform by construction (helps the compiler)
 
   // ---- work item: sink tiles of every head first, then head-major with ascending KV tile ----
   int hk, b, j;
@@ -219,11 +221,12 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           tma_load_3d(sK + s * SLAB_KV, &tmK, bar_kv, s * 64, k0, bhk);
           tma_load_3d(sV + s * SLAB_KV, &tmV, bar_kv, s * 64, k0, bhk);
         }
+        int st = 0, g = 0, t_in = 0;   // stage, head of the group, position in I_h(j): kept incrementally
+        uint32_t ph_e = 0;             // parity of the "stage empty" wait (the first NST steps need none)
         for (int n = 0; n < N && ok; ++n) {
-          const int st = n % NST;
-          if (n >= NST) ok = mbar_wait(bar_ld_empty + st, ((n / NST) - 1) & 1, a.status);
+          if (n >= NST) ok = mbar_wait(bar_ld_empty + st, ph_e, a.status);
           if (!ok) break;
-          const int g = n / cnt, i = cowa_bwd_tile_at(rg, n % cnt);
+          const int i = cowa_bwd_tile_at(rg, t_in);
           const int bhq = b * a.Hq + hk * a.G + g, q0 = i * BQS;
           uint8_t* sQ = sStage + st * SM::kStage;
           uint8_t* sdO = sQ + SM::kQS;
@@ -234,94 +237,121 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           }
           bulk_load_1d(sVec + st * 128, a.lse2 + (size_t)bhq * a.Tpad + q0, 256, bar_ld_full + st);
           bulk_load_1d(sVec + st * 128 + 64, a.delta + (size_t)bhq * a.Tpad + q0, 256, bar_ld_full + st);
+          if (++t_in == cnt) { t_in = 0; ++g; }
+          if (++st == NST) { st = 0; if (n >= NST) ph_e ^= 1; }
         }
       }
     } else if (warp == 1) {
       // ================= MMA issuer =================
-      if (lane == 0 && N > 0) {
-        // Descriptors are built once per operand base; a byte offset o inside the tile is added as o >> 4
-        // to the descriptor's address field (the tiles never cross the field's range).
-        const uint64_t dK_k = smem_desc_sw128(smem_u32(sK), 16, 1024);                           // K, K-major (A of S^T)
-        const uint64_t dV_k = smem_desc_sw128(smem_u32(sV), 16, 1024);                           // V, K-major (A of dP^T)
-        const uint64_t dK_mn = smem_desc_sw128(smem_u32(sK), D == 128 ? SLAB_KV : 0, 1024);      // K^T, MN-major (A of dQ^T)
-        auto gemm_st = [&](uint32_t d_col, uint64_t dA, const uint8_t* sB) {  // [128 x 64] = A[128xD] B[64xD]^T
-          const uint64_t dB = smem_desc_sw128(smem_u32(sB), 16, 1024);
+      // The whole warp runs this loop (uniform control flow, so that descriptors and counters stay in
+      // uniform registers); only the elected lane executes the tcgen05 instructions.  Everything that
+      // can be computed once is: descriptor of every operand base, stage and parity bookkeeping is
+      // incremental, and the loop body is instantiated for both TMEM buffers.
+      if (N > 0) {
+        const bool lead = elect_one();
+        const uint32_t tb = tmem_base;
+        // Descriptors: a byte offset o inside a tile is added as o >> 4 to the address field (bits 0-13);
+        // no tile crosses the field's range, so the 64-bit add never carries out of it.
+        const uint64_t dK_k = smem_desc_sw128(smem_u32(sK), 16, 1024);                       // K, K-major (A of S^T)
+        const uint64_t dV_k = smem_desc_sw128(smem_u32(sV), 16, 1024);                       // V, K-major (A of dP^T)
+        const uint64_t dK_mn = smem_desc_sw128(smem_u32(sK), D == 128 ? SLAB_KV : 0, 1024);  // K^T, MN-major (A of dQ^T)
+        const uint64_t dQ_k0 = smem_desc_sw128(smem_u32(sStage), 16, 1024);                  // Q of stage 0, K-major (B of S^T)
+        const uint64_t dO_k0 = smem_desc_sw128(smem_u32(sStage) + SM::kQS, 16, 1024);        // dO of stage 0, K-major (B of dP^T)
+        const uint64_t dQ_mn0 = smem_desc_sw128(smem_u32(sStage), SLAB_QS, 1024);            // Q, MN-major (B of dK)
+        const uint64_t dO_mn0 = smem_desc_sw128(smem_u32(sStage) + SM::kQS, SLAB_QS, 1024);  // dO, MN-major (B of dV)
+        const uint64_t dDS0 = smem_desc_sw128(smem_u32(sDS), 0, 1024);                       // dS^T, MN-major (B of dQ^T)
+        constexpr uint32_t kStage16 = SM::kStage >> 4, kDS16 = SM::kDS >> 4;
+
+        auto gemm_st = [&](uint32_t d_col, uint64_t dA, uint64_t dB) {  // [128 x 64] = A[128 x D] B[64 x D]^T
+          if (lead) {
 #pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk) {
-            const uint32_t oa = (kk / 4) * SLAB_KV + (kk % 4) * 32, ob = (kk / 4) * SLAB_QS + (kk % 4) * 32;
-            mma_ss(tmem_base + d_col, dA + (oa >> 4), dB + (ob >> 4), ID_ST, kk > 0);
+            for (int kk = 0; kk < D / 16; ++kk)
+              mma_ss(tb + d_col, dA + (((kk / 4) * SLAB_KV + (kk % 4) * 32) >> 4),
+                     dB + (((kk / 4) * SLAB_QS + (kk % 4) * 32) >> 4), ID_ST, kk > 0);
           }
         };
-        auto gemm_acc = [&](uint32_t d_col, uint32_t a_col, const uint8_t* sB, bool first) {  // [128 x D] += A^T-in-TMEM B
-          const uint64_t dB = smem_desc_sw128(smem_u32(sB), SLAB_QS, 1024);
+        auto gemm_acc = [&](uint32_t d_col, uint32_t a_col, uint64_t dB, uint32_t acc_first) {  // [128 x D] += A(TMEM) B
+          if (lead) {
 #pragma unroll
-          for (int kk = 0; kk < BQS / 16; ++kk)
-            mma_ts(tmem_base + d_col, tmem_base + a_col + kk * 8, dB + ((kk * 2048) >> 4), ID_ACC,
-                   (!first || kk > 0) ? 1u : 0u);
+            for (int kk = 0; kk < BQS / 16; ++kk)
+              mma_ts(tb + d_col, tb + a_col + kk * 8, dB + ((kk * 2048) >> 4), ID_ACC, kk > 0 ? 1u : acc_first);
+          }
         };
-        auto gemm_dq = [&](uint32_t d_col, const uint8_t* sB) {  // dQ^T[D x 64] = K^T dS^T
-          const uint64_t dB = smem_desc_sw128(smem_u32(sB), 0, 1024);
+        auto gemm_dq = [&](uint32_t d_col, uint64_t dB) {  // dQ^T[D x 64] = K^T dS^T
+          if (lead) {
 #pragma unroll
-          for (int kk = 0; kk < BKV / 16; ++kk)
-            mma_ss(tmem_base + d_col, dK_mn + ((kk * 2048) >> 4), dB + ((kk * 2048) >> 4), ID_DQ, kk > 0);
+            for (int kk = 0; kk < BKV / 16; ++kk)
+              mma_ss(tb + d_col, dK_mn + ((kk * 2048) >> 4), dB + ((kk * 2048) >> 4), ID_DQ, kk > 0);
+          }
         };
+        auto commit = [&](uint64_t* bar) {
+          if (lead) mma_commit(bar);
+        };
+
         ok = mbar_wait(bar_kv, 0, a.status);
         // prologue: S^T(0), dP^T(0), S^T(1)
         ok = ok && mbar_wait(bar_ld_full + 0, 0, a.status);
         if (ok) {
           tc_fence_after();
-          gemm_st(cS0, dK_k, sStage);
-          mma_commit(bar_s_full + 0);
-          gemm_st(cDP0, dV_k, sStage + SM::kQS);
-          mma_commit(bar_dp_full + 0);
+          gemm_st(cS0, dK_k, dQ_k0);
+          commit(bar_s_full + 0);
+          gemm_st(cDP0, dV_k, dO_k0);
+          commit(bar_dp_full + 0);
         }
         if (ok && N > 1) {
           ok = mbar_wait(bar_ld_full + 1, 0, a.status);
           if (ok) {
             tc_fence_after();
-            gemm_st(cS0 + 64, dK_k, sStage + SM::kStage);
-            mma_commit(bar_s_full + 1);
+            gemm_st(cS0 + 64, dK_k, dQ_k0 + kStage16);
+            commit(bar_s_full + 1);
           }
         }
         // Step n uses TMEM buffer b = n & 1 (the two compute warpgroups alternate steps).  Issue order:
         //   dV(n) | dP^T(n+1) | dK(n) | dQ^T(n) | S^T(n+2)
         // so that every wait below is for something produced about one step earlier.
-        for (int n = 0; n < N && ok; ++n) {
-          const int st = n % NST, b_ = n & 1;
-          const uint32_t par = (n >> 1) & 1;
-          uint8_t* sQ = sStage + st * SM::kStage;
-          uint8_t* sdO = sQ + SM::kQS;
-          const uint32_t sbuf = cS0 + b_ * 64, dpbuf = cDP0 + b_ * 64;
+        int st = 0, st1 = (N > 1) ? 1 : 0, st2 = 2 % NST;    // stages of steps n, n+1, n+2
+        uint32_t ph2 = (2 / NST) & 1;                        // parity of the load that fills stage st2 for step n+2
+        uint32_t par = 0;                                    // (n >> 1) & 1
+        auto body = [&](int n, auto B_) {
+          constexpr int b_ = decltype(B_)::value;
+          constexpr uint32_t sbuf = cS0 + b_ * 64, dpbuf = cDP0 + b_ * 64, dpother = cDP0 + (b_ ^ 1) * 64;
           ok = mbar_wait(bar_p_ready + b_, par, a.status);
-          if (!ok) break;
+          if (!ok) return;
           tc_fence_after();
-          gemm_acc(cDV, sbuf, sdO, n == 0);                // dV += P^T dO
-          if (n + 1 < N) {                                 // dP^T(n+1) into the other buffer, once dQ^T(n-1) has left it
+          gemm_acc(cDV, sbuf, dO_mn0 + st * kStage16, n > 0 ? 1u : 0u);     // dV += P^T dO
+          if (n + 1 < N) {                                                  // dP^T(n+1), once dQ^T(n-1) has left its buffer
             if (n >= 1) {
               ok = mbar_wait(bar_dq_free + (b_ ^ 1), ((n - 1) >> 1) & 1, a.status);
-              if (!ok) break;
+              if (!ok) return;
               tc_fence_after();
             }
-            gemm_st(cDP0 + (b_ ^ 1) * 64, dV_k, sStage + ((n + 1) % NST) * SM::kStage + SM::kQS);
-            mma_commit(bar_dp_full + (b_ ^ 1));
+            gemm_st(dpother, dV_k, dO_k0 + st1 * kStage16);
+            commit(bar_dp_full + (b_ ^ 1));
           }
           ok = mbar_wait(bar_ds_ready + b_, par, a.status);
-          if (!ok) break;
+          if (!ok) return;
           tc_fence_after();
-          gemm_acc(cDK, sbuf + 32, sQ, n == 0);            // dK += dS^T Q
-          mma_commit(bar_ld_empty + st);
-          gemm_dq(dpbuf, sDS + b_ * SM::kDS);              // dQ^T = K^T dS^T, over the consumed dP^T(n)
-          mma_commit(bar_dq_full + b_);
-          if (n + 2 < N) {                                 // S^T(n+2) into the buffer that P^T(n), dS^T(n) just left
-            const int s2 = (n + 2) % NST;
-            ok = mbar_wait(bar_ld_full + s2, ((n + 2) / NST) & 1, a.status);
-            if (!ok) break;
+          gemm_acc(cDK, sbuf + 32, dQ_mn0 + st * kStage16, n > 0 ? 1u : 0u);  // dK += dS^T Q
+          commit(bar_ld_empty + st);
+          gemm_dq(dpbuf, dDS0 + b_ * kDS16);                                // dQ^T = K^T dS^T over the consumed dP^T(n)
+          commit(bar_dq_full + b_);
+          if (n + 2 < N) {                                                  // S^T(n+2) into the buffer P^T(n), dS^T(n) just left
+            ok = mbar_wait(bar_ld_full + st2, ph2, a.status);
+            if (!ok) return;
             tc_fence_after();
-            gemm_st(sbuf, dK_k, sStage + s2 * SM::kStage);
-            mma_commit(bar_s_full + b_);
+            gemm_st(sbuf, dK_k, dQ_k0 + st2 * kStage16);
+            commit(bar_s_full + b_);
           }
+          // advance the bookkeeping to step n+1
+          st = st1; st1 = st2;
+          if (++st2 == NST) { st2 = 0; ph2 ^= 1; }
+          if (b_ == 1) par ^= 1;
+        };
+        for (int n = 0; n < N && ok; n += 2) {
+          body(n, std::integral_constant<int, 0>{});
+          if (n + 1 < N && ok) body(n + 1, std::integral_constant<int, 1>{});
         }
-        mma_commit(bar_done);
+        commit(bar_done);
       }
     }
   } else if (warp < 12) {
@@ -336,10 +366,10 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const long long kpos = (long long)kcol - off;  // first causal query of this key
       const float2 sc2 = make_float2(a.scale_log2, a.scale_log2);
       uint8_t* ds_row = sDS + wg * SM::kDS + r * 128;
+      int st = wg % NST, t_in = cnt > 0 ? wg % cnt : 0;   // stage and position in I_h(j) of this warpgroup's next step
+      uint32_t ph_l = (wg / NST) & 1, par = 0;
       for (int n = wg; n < N && ok; n += 2) {
-        const int st = n % NST;
-        const uint32_t par = (n >> 1) & 1;
-        const int i = cowa_bwd_tile_at(rg, n % cnt);
+        const int i = cowa_bwd_tile_at(rg, t_in);
         const int q0 = i * BQS;
         const bool full = cowa_tile_full(w, q0, BQS, k0, BKV, off, a.Nq, a.Nk);
         uint32_t mk[2] = {0xFFFFFFFFu, 0xFFFFFFFFu};
@@ -357,7 +387,7 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         }
         const float* lse2 = sVec + st * 128;
         const float* dlt = lse2 + 64;
-        ok = mbar_wait(bar_ld_full + st, (n / NST) & 1, a.status);
+        ok = mbar_wait(bar_ld_full + st, ph_l, a.status);
         ok = ok && mbar_wait(bar_s_full + wg, par, a.status);
         if (!ok) break;
         tc_fence_after();
@@ -413,6 +443,9 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         tc_fence_before();
         fence_proxy_async_smem();
         mbar_arrive(bar_ds_ready + wg);
+        par ^= 1;
+        st += 2; if (st >= NST) { st -= NST; ph_l ^= 1; }
+        t_in += 2; if (t_in >= cnt) t_in -= cnt; if (t_in >= cnt) t_in %= cnt;
       }
       if (wg == 0) store_grad(true);
     }
@@ -423,9 +456,11 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const int d = (warp & 3) * 32 + lane;
       const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
       const bool issuer = (d == 0);
+      int g = 0, t_in = 0;
       for (int n = 0; n < N && ok; ++n) {
-        const int g = n / cnt, i = cowa_bwd_tile_at(rg, n % cnt);
+        const int i = cowa_bwd_tile_at(rg, t_in);
         const int bhq = b * a.Hq + hk * a.G + g, q0 = i * BQS;
+        if (++t_in == cnt) { t_in = 0; ++g; }
         ok = mbar_wait(bar_dq_full + (n & 1), (n >> 1) & 1, a.status);
         if (!ok) break;
         tc_fence_after();
