@@ -78,7 +78,8 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   uint64_t* bar_pv = bars + 9;  //     O += P V of a step has completed
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 10);
 
-  const int tid = threadIdx.x, warp = tid >> 5;
+  const int tid = threadIdx.x;
+  const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);  // warp-uniform by construction
 
   // ---- work item (heaviest QO tiles first; the group's heads adjacent) ----
   int idx = blockIdx.x;
@@ -118,45 +119,60 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   bool ok = true;  // false once a bounded wait ran out; every role then falls through to the teardown
 
   if (warp == 4) {
-    // ======================= control: TMA loads and MMA issue (one lane) =======================
-    if (tid == 128 && nt > 0) {
-      prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV);
+    // ======================= control: TMA loads and MMA issue =======================
+    // The whole warp runs the loop (uniform control flow keeps descriptors and counters in uniform
+    // registers); only the elected lane executes the TMA and tcgen05 instructions.
+    if (nt > 0) {
+      const bool lead = elect_one();
+      const uint32_t tb = tmem_base;
+      const uint64_t dQ = smem_desc_sw128(smem_u32(sQ), 16, 1024);                 // Q, K-major (A of S)
+      const uint64_t dK0 = smem_desc_sw128(smem_u32(sK), 16, 1024);                // K buffer 0, K-major (B of S)
+      const uint64_t dV0 = smem_desc_sw128(smem_u32(sV), SLAB_K, 1024);            // V buffer 0, MN-major (B of O)
+      constexpr uint32_t kKV16 = SM::kKV >> 4;
       auto load_k = [&](int t) {
-        const int j = cowa_fwd_tile_at(rg, t);
-        uint8_t* dst = sK + (t & 1) * SM::kKV;
-        mbar_expect_tx(bar_k + (t & 1), SM::kKV);
-        for (int s = 0; s < NSLAB; ++s) tma_load_3d(dst + s * SLAB_K, &tmK, bar_k + (t & 1), s * 64, j * BK, bhk);
+        if (lead) {
+          const int j = cowa_fwd_tile_at(rg, t);
+          uint8_t* dst = sK + (t & 1) * SM::kKV;
+          mbar_expect_tx(bar_k + (t & 1), SM::kKV);
+          for (int s = 0; s < NSLAB; ++s) tma_load_3d(dst + s * SLAB_K, &tmK, bar_k + (t & 1), s * 64, j * BK, bhk);
+        }
       };
       auto load_v = [&](int t) {
-        const int j = cowa_fwd_tile_at(rg, t);
-        uint8_t* dst = sV + (t & 1) * SM::kKV;
-        mbar_expect_tx(bar_v + (t & 1), SM::kKV);
-        for (int s = 0; s < NSLAB; ++s) tma_load_3d(dst + s * SLAB_K, &tmV, bar_v + (t & 1), s * 64, j * BK, bhk);
+        if (lead) {
+          const int j = cowa_fwd_tile_at(rg, t);
+          uint8_t* dst = sV + (t & 1) * SM::kKV;
+          mbar_expect_tx(bar_v + (t & 1), SM::kKV);
+          for (int s = 0; s < NSLAB; ++s) tma_load_3d(dst + s * SLAB_K, &tmV, bar_v + (t & 1), s * 64, j * BK, bhk);
+        }
       };
-      const uint64_t dQ = smem_desc_sw128(smem_u32(sQ), 16, 1024);
-      auto issue_s = [&](int t) {  // S(t) = Q K(t)^T into buffer t & 1
-        const uint64_t dK = smem_desc_sw128(smem_u32(sK + (t & 1) * SM::kKV), 16, 1024);
+      auto issue_s = [&](int buf) {  // S = Q K^T into TMEM buffer buf from K buffer buf
+        if (lead) {
+          const uint64_t dK = dK0 + buf * kKV16;
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk)
-          mma_ss(tmem_base + (t & 1) * 64, dQ + (((kk / 4) * SLAB_Q + (kk % 4) * 32) >> 4),
-                 dK + (((kk / 4) * SLAB_K + (kk % 4) * 32) >> 4), IDESC_S, kk > 0);
-        mma_commit(bar_s + (t & 1));
+          for (int kk = 0; kk < D / 16; ++kk)
+            mma_ss(tb + buf * 64, dQ + (((kk / 4) * SLAB_Q + (kk % 4) * 32) >> 4),
+                   dK + (((kk / 4) * SLAB_K + (kk % 4) * 32) >> 4), IDESC_S, kk > 0);
+          mma_commit(bar_s + buf);
+        }
       };
-      mbar_expect_tx(bar_q, SM::kQ);
-      for (int s = 0; s < NSLAB; ++s) tma_load_3d(sQ + s * SLAB_Q, &tmQ, bar_q, s * 64, q0, bhq);
+      if (lead) {
+        prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV);
+        mbar_expect_tx(bar_q, SM::kQ);
+        for (int s = 0; s < NSLAB; ++s) tma_load_3d(sQ + s * SLAB_Q, &tmQ, bar_q, s * 64, q0, bhq);
+      }
       load_k(0);
       if (nt > 1) load_k(1);
       load_v(0);
       ok = mbar_wait(bar_q, 0, a.status) && mbar_wait(bar_k, 0, a.status);
       if (ok) { tc_fence_after(); issue_s(0); }
+      uint32_t par = 0;  // (t >> 1) & 1
       for (int t = 0; t < nt && ok; ++t) {
         const int b_ = t & 1;
-        const uint32_t par = (t >> 1) & 1;
         if (t + 1 < nt) {  // S(t+1): its buffer last held P(t-1), whose product was issued before this one
-          ok = mbar_wait(bar_k + (b_ ^ 1), ((t + 1) >> 1) & 1, a.status);
+          ok = mbar_wait(bar_k + (b_ ^ 1), b_ ? (par ^ 1) : par, a.status);
           if (!ok) break;
           tc_fence_after();
-          issue_s(t + 1);
+          issue_s(b_ ^ 1);
         }
         if (t + 2 < nt) {  // K(t+2) over K(t), once S(t) has been computed
           ok = mbar_wait(bar_s + b_, par, a.status);
@@ -171,12 +187,14 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         ok = mbar_wait(bar_p + b_, par, a.status) && mbar_wait(bar_v + b_, par, a.status);
         if (!ok) break;
         tc_fence_after();
-        const uint64_t dV = smem_desc_sw128(smem_u32(sV + b_ * SM::kKV), SLAB_K, 1024);
+        if (lead) {
+          const uint64_t dV = dV0 + b_ * kKV16;
 #pragma unroll
-        for (int kk = 0; kk < BK / 16; ++kk)
-          mma_ts(tmem_base + cO, tmem_base + b_ * 64 + kk * 8, dV + ((kk * 2048) >> 4), IDESC_O,
-                 (t > 0 || kk > 0) ? 1u : 0u);
-        mma_commit(bar_pv);
+          for (int kk = 0; kk < BK / 16; ++kk)
+            mma_ts(tb + cO, tb + b_ * 64 + kk * 8, dV + ((kk * 2048) >> 4), IDESC_O, (t > 0 || kk > 0) ? 1u : 0u);
+          mma_commit(bar_pv);
+        }
+        if (b_) par ^= 1;
       }
     }
   } else {
