@@ -59,10 +59,10 @@ struct BwdSmem {
   static constexpr int kDS = BKV * BQS * 2;    // dS^T tile (bf16)
   static constexpr int oK = 0, oV = kKV, oStage = 2 * kKV, oDS = oStage + NST * kStage;
   static constexpr int oVec = oDS + 2 * kDS;   // per stage: 64 floats lse2, 64 floats delta
-  static constexpr int oDQ = oVec + NST * 512;  // dQ staging: 32 query rows x D fp32
+  static constexpr int oDQ = oVec + NST * 512;  // dQ staging: two tiles of 32 query rows x D fp32
   static constexpr int kDQ = 32 * D * 4;
-  static constexpr int oBar = oDQ + kDQ;
-  static constexpr int kBytes = oBar + 256 + 1024;
+  static constexpr int oBar = oDQ + 2 * kDQ;
+  static constexpr int kBytes = oBar + 256 + 1024;  // barriers + alignment slack; 232192 B at D = 128 (limit 232448)
 };
 
 __device__ __forceinline__ void bulk_load_1d(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
@@ -472,16 +472,17 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         mbar_arrive(bar_dq_free + (n & 1));
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) {
-          if (issuer) tma_wait_group_read<0>();  // the previous reduction has finished reading the staging tile
+          float* stage = sDQ + hf * (SM::kDQ / 4);
+          if (issuer) tma_wait_group_read<1>();  // the reduction issued from this tile one step ago has read it
           wg_sync(3);
           if (d < D) {
 #pragma unroll
-            for (int c = 0; c < 32; ++c) sDQ[c * D + d] = __uint_as_float(v[hf][c]) * a.scale;
+            for (int c = 0; c < 32; ++c) stage[c * D + d] = __uint_as_float(v[hf][c]) * a.scale;
           }
           fence_proxy_async_smem();
           wg_sync(3);
           if (issuer) {
-            tma_reduce_add_3d(&tmdQ, sDQ, 0, q0 + hf * 32, bhq);
+            tma_reduce_add_3d(&tmdQ, stage, 0, q0 + hf * 32, bhq);
             tma_commit_group();
           }
         }
