@@ -72,6 +72,14 @@ typedef struct {
 int cowa_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
              int B, int T, int Hq, int Hkv, int D, const cowa_params_t* p, void* stream);
 
+/* Inference prefill, also chunked prefill into an existing cache: the same forward operator with
+ * N_q <= N_k (Sec. 2.3 "Forward execution"; Sec. 2.1: query i_q sits at key position i_q + (N_k - N_q),
+ * Eq. fwa_distance, and the windows are built from N_k).
+ *   q [B,Hq,Nq,D]; k,v [B,Hkv,Nk,D] in; o [B,Hq,Nq,D] bf16 and lse [B,Hq,Nq] fp32 out.
+ * Every sequence of the batch has the same Nq and Nk.  cowa_fwd is this call with Nq = Nk = T. */
+int cowa_prefill(const void* q, const void* k, const void* v, void* o, float* lse,
+                 int B, int Nq, int Nk, int Hq, int Hkv, int D, const cowa_params_t* p, void* stream);
+
 /* Training backward, Algorithm 2: exact gradient of cowa_fwd.
  *   in: q,k,v,o,lse as produced by cowa_fwd, d_o [B,Hq,T,D];
  *   out: dq [B,Hq,T,D], dk,dv [B,Hkv,T,D] bf16 (fully overwritten).

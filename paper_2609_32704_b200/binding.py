@@ -48,6 +48,8 @@ def lib():
         pp = C.POINTER(Params)
         L.cowa_fwd.argtypes = [vp] * 5 + [i32] * 5 + [pp, vp]
         L.cowa_fwd.restype = i32
+        L.cowa_prefill.argtypes = [vp] * 5 + [i32] * 6 + [pp, vp]
+        L.cowa_prefill.restype = i32
         L.cowa_bwd.argtypes = [vp] * 9 + [i32] * 5 + [pp, vp, sz, vp]
         L.cowa_bwd.restype = i32
         L.cowa_decode.argtypes = [vp] * 6 + [i32] * 5 + [pp, vp, sz, vp]
@@ -125,6 +127,18 @@ def cowa_fwd(q, k, v, o, lse, params):
     Hkv = k.shape[1]
     _check(lib().cowa_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), B, T, Hq, Hkv, D,
                           C.byref(params), _stream()), "cowa_fwd")
+
+
+def cowa_prefill(q, k, v, o, lse, params):
+    """Forward with N_q <= N_k (bottom-right aligned): q [B,Hq,Nq,D], k/v [B,Hkv,Nk,D] -> o, lse [B,Hq,Nq]."""
+    import torch
+    for t, n in ((q, "q"), (k, "k"), (v, "v"), (o, "o")):
+        _need(t, torch.bfloat16, n)
+    _need(lse, torch.float32, "lse")
+    B, Hq, Nq, D = q.shape
+    Hkv, Nk = k.shape[1], k.shape[2]
+    _check(lib().cowa_prefill(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), B, Nq, Nk, Hq, Hkv, D,
+                              C.byref(params), _stream()), "cowa_prefill")
 
 
 def cowa_bwd_workspace_bytes(B, T, Hq, Hkv, D, params):

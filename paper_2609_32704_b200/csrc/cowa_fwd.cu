@@ -340,24 +340,24 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 }
 
 template <int D>
-int launch_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int T, int Hq, int Hkv,
-               const cowa_params_t* p, const CowaHeadWindows& hw, cudaStream_t st) {
+int launch_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Nq, int Nk, int Hq,
+               int Hkv, const cowa_params_t* p, const CowaHeadWindows& hw, cudaStream_t st) {
   CUtensorMap mq, mk, mv, mo;
   int rc;
-  if ((rc = cowa::make_tensor_map_3d(&mq, q, cowa::MapType::BF16, D, T, (long long)B * Hq, 64, BQ))) return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mk, k, cowa::MapType::BF16, D, T, (long long)B * Hkv, 64, BK))) return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mv, v, cowa::MapType::BF16, D, T, (long long)B * Hkv, 64, BK))) return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mo, o, cowa::MapType::BF16, D, T, (long long)B * Hq, 64, BQ))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mq, q, cowa::MapType::BF16, D, Nq, (long long)B * Hq, 64, BQ))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mk, k, cowa::MapType::BF16, D, Nk, (long long)B * Hkv, 64, BK))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mv, v, cowa::MapType::BF16, D, Nk, (long long)B * Hkv, 64, BK))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mo, o, cowa::MapType::BF16, D, Nq, (long long)B * Hq, 64, BQ))) return rc;
   FwdArgs a;
   a.lse = lse;
   a.status = cowa::device_status_word();
   if (!a.status) return COWA_ERR_CUDA;
-  a.B = B; a.Nq = T; a.Nk = T; a.Hq = Hq; a.Hkv = Hkv; a.G = Hq / Hkv;
+  a.B = B; a.Nq = Nq; a.Nk = Nk; a.Hq = Hq; a.Hkv = Hkv; a.G = Hq / Hkv;
   a.scale_log2 = p->softmax_scale * 1.4426950408889634f;
   a.wins = hw;
   COWA_CUDA_TRY(cudaFuncSetAttribute(cowa_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      FwdSmem<D>::kBytes));
-  const long long nblocks = (long long)((T + BQ - 1) / BQ) * B * Hq;
+  const long long nblocks = (long long)((Nq + BQ - 1) / BQ) * B * Hq;
   if (nblocks > 0x7FFFFFFFll) return COWA_ERR_UNSUPPORTED;
   cowa_fwd_kernel<D><<<(unsigned)nblocks, kFwdThreads, FwdSmem<D>::kBytes, st>>>(mq, mk, mv, mo, a);
   COWA_CUDA_TRY(cudaGetLastError());
@@ -366,18 +366,27 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
 
 }  // namespace
 
-extern "C" int cowa_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int T, int Hq,
-                        int Hkv, int D, const cowa_params_t* p, void* stream) {
+extern "C" {
+
+int cowa_prefill(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Nq, int Nk, int Hq,
+                 int Hkv, int D, const cowa_params_t* p, void* stream) {
   if (!q || !k || !v || !o || !lse || !p) return COWA_ERR_INVALID_ARG;
-  if (B <= 0 || T <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0) return COWA_ERR_INVALID_ARG;
+  if (B <= 0 || Nq <= 0 || Nk < Nq || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0) return COWA_ERR_INVALID_ARG;
   if (!(p->softmax_scale > 0.f)) return COWA_ERR_INVALID_ARG;
   if (D != 64 && D != 128) return COWA_ERR_UNSUPPORTED;
   if (!cowa::aligned16(q) || !cowa::aligned16(k) || !cowa::aligned16(v) || !cowa::aligned16(o))
     return COWA_ERR_MISALIGNED;
   CowaHeadWindows hw;
-  int rc = cowa::resolve_windows(T, Hkv, p, &hw);
+  int rc = cowa::resolve_windows(Nk, Hkv, p, &hw);
   if (rc != COWA_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  return D == 128 ? launch_fwd<128>(q, k, v, o, lse, B, T, Hq, Hkv, p, hw, st)
-                  : launch_fwd<64>(q, k, v, o, lse, B, T, Hq, Hkv, p, hw, st);
+  return D == 128 ? launch_fwd<128>(q, k, v, o, lse, B, Nq, Nk, Hq, Hkv, p, hw, st)
+                  : launch_fwd<64>(q, k, v, o, lse, B, Nq, Nk, Hq, Hkv, p, hw, st);
 }
+
+int cowa_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int T, int Hq, int Hkv, int D,
+             const cowa_params_t* p, void* stream) {
+  return cowa_prefill(q, k, v, o, lse, B, T, T, Hq, Hkv, D, p, stream);
+}
+
+}  // extern "C"

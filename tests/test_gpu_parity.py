@@ -114,6 +114,33 @@ def test_fwd_8k_config_sampled_heads():
     check("dup o", o[0, 13].float().cpu().numpy(), o_ref)
 
 
+# ------------------------------------------------------------------ prefill (N_q <= N_k)
+
+@pytest.mark.parametrize("B,Nq,Nk,Hq,Hkv,D,sink,local", [
+    (1, 256, 1024, 4, 2, 128, 16, 100),    # a chunk appended to an existing cache
+    (2, 100, 777, 8, 2, 64, 5, 60),        # ragged sizes
+    (1, 1, 2000, 4, 2, 128, 32, 200),      # one query: the decode case through the forward kernel
+    (1, 513, 514, 2, 1, 128, 0, 7),        # off = 1, H_k = 1
+    (1, 300, 5000, 8, 4, 128, 64, 256),    # far bands clipped at the first keys
+])
+def test_prefill_shapes(B, Nq, Nk, Hq, Hkv, D, sink, local):
+    q, _, _, _ = cowa_inputs.make_train_inputs(53, B, Nq, Hq, Hkv, D)
+    _, k, v, _ = cowa_inputs.make_train_inputs(54, B, Nk, Hq, Hkv, D)
+    scale = cowa_inputs.softmax_scale(D)
+    params = cowa.make_params(sink=sink, local=local, softmax_scale=scale)
+    o = torch.full_like(q, float("nan")).to(DEV)
+    lse = torch.full((B, Hq, Nq), float("nan"), dtype=torch.float32, device=DEV)
+    cowa.cowa_prefill(q.to(DEV), k.to(DEV), v.to(DEV), o, lse, params)
+    torch.cuda.synchronize()
+    cowa.cowa_check_device_status()
+    ws = orc.default_windows(Nk, Hkv, sink, local)
+    f = cowa_inputs.to_f64
+    for b in range(B):
+        o_ref, lse_ref = orc.forward(f(q[b]), f(k[b]), f(v[b]), ws, scale)
+        check(f"prefill lse[b={b}]", lse[b].cpu().numpy(), lse_ref, TOL_LSE, TOL_LSE)
+        check(f"prefill o[b={b}]", o[b].float().cpu().numpy(), o_ref)
+
+
 # ------------------------------------------------------------------ backward
 
 def run_fwd_bwd(q, k, v, d_o, params):
