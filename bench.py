@@ -383,8 +383,8 @@ def run_cuda(args):
         dom, dom_flops, dom_ms = "cowa_fwd_kernel<128>", fwd_flops, fwd_ms
     peak_tf = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
     achieved = dom_flops / dom_ms / 1e9
-    # DRAM bytes per launch of the dominant kernel at the 128K workload, from the one-pass ncu capture
-    # summarised in profiles/launch_list_bench_128k.md (dram__bytes_read.sum + dram__bytes_write.sum).
+    # DRAM bytes per launch of the dominant kernel at the 128K workload: dram__bytes_read.sum +
+    # dram__bytes_write.sum of a one-pass ncu capture of this same command.
     traffic_128k = {"cowa_bwd_kernel<128>": 12.876e9 + 6.633e9, "cowa_fwd_kernel<128>": 10.145e9 + 1.054e9}
     roofline = {"kernel": dom, "bound": "tensor", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s",
                 "frac": achieved / peak_tf, "peak_source": f"{peak_src} bf16 sustained (kernel timed inside a long step)",
