@@ -10,6 +10,11 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200)")
+    # The tests call the C-ABI library; build it in-tree (nvcc cross-compiles without a GPU) when a fresh
+    # checkout has not done so yet.
+    from paper_2609_32704_b200.build import LIB_PATH, build_library
+    if not os.path.exists(LIB_PATH):
+        build_library()
 
 
 def read_golden(name):
