@@ -4,15 +4,16 @@
 // online-softmax states are merged afterwards.
 //
 // HBM-bound: every visible K and V row is read exactly once, with 128-bit loads, straight
-// into registers.  Per (sequence, KV head, split) one 128-thread block:
+// into registers.  Per (sequence, KV head, split) one 128-thread block, 5 blocks per SM:
 //   1. scores:  each warp takes 16 visible rows at a time; K rows are loaded as the A
 //      fragment of mma.sync m16n8k16 (bf16, fp32 accumulate), the group's query vectors are
 //      the B fragment.  The contraction index is permuted identically on both operands so
 //      that every thread's loads are 16-byte vectors.  Scores (log2 units) go to shared memory.
 //   2. block-wide max / exp2 / sum per QO head (no running rescale: the split's scores are
 //      all in shared memory before any V row is touched).
-//   3. values:  thread = (8-wide slice of D, row subgroup); fp32 FMAs over the split's V rows
-//      with the probabilities broadcast from shared memory; row subgroups reduced in shared
+//   3. values:  again mma.sync m16n8k16, O^T += V^T P^T with 16 visible rows per instruction; V rows are
+//      loaded with 16-byte vectors and neighbouring rows are paired with byte permutes (the d index is
+//      permuted inside the fragment and restored on output); the four warps' partial sums meet in shared
 //      memory; un-normalised partial (o, m, l) written to the workspace.
 // A second kernel merges the splits (log-sum-exp combine with warp shuffles).
 #include <cuda_bf16.h>
@@ -23,6 +24,7 @@ namespace {
 
 constexpr int kThreads = 128;
 constexpr int kChunkCap = 1024;  // max visible rows per split (scores of a split live in shared memory)
+constexpr int kScStride = kChunkCap + 8;  // row stride of the score array: heads land in different banks
 
 // Scratch of cowa_decode_static: lives in the library's device image, so every GPU that loads the
 // library keeps these bytes reserved until the process exits.
@@ -85,21 +87,14 @@ __device__ __forceinline__ uint4 ldg128(const void* p) {
   return r;
 }
 
-__device__ __forceinline__ float bf16lo(uint32_t x) { return __uint_as_float(x << 16); }
-__device__ __forceinline__ float bf16hi(uint32_t x) { return __uint_as_float(x & 0xffff0000u); }
-
 template <int D, int G>
-#ifndef COWA_DEC_MINB
-#define COWA_DEC_MINB 7
-#endif
-__global__ void __launch_bounds__(kThreads, COWA_DEC_MINB) cowa_decode_split_kernel(const DecodeArgs a) {
+// 5 blocks per SM (up to 102 registers, no spills) measured best: fewer, longer splits than at 7 per SM
+__global__ void __launch_bounds__(kThreads, 5) cowa_decode_split_kernel(const DecodeArgs a) {
   static_assert(D == 64 || D == 128, "head dim");
   static_assert(G >= 1 && G <= 8, "group size per mma n-tile");
-  constexpr int DC = D / 8;           // 16-byte slices per row
-  constexpr int RP = kThreads / DC;   // rows handled in parallel in the value phase
   constexpr int KC = D / 32;          // 32-wide d chunks (two k16 steps each)
 
-  __shared__ __align__(16) float sc[G * kChunkCap];  // scores, later the value-phase reduction buffer
+  __shared__ __align__(16) float sc[G * kScStride];  // scores, later the value-phase reduction buffer
   __shared__ float m_s[G], l_s[G];
 
   const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
@@ -168,12 +163,12 @@ __global__ void __launch_bounds__(kThreads, COWA_DEC_MINB) cowa_decode_split_ker
       // c[0],c[1]: row rA, heads 2t, 2t+1;  c[2],c[3]: row rB
       const int h0 = 2 * t, h1 = 2 * t + 1;
       if (rA < clen) {
-        if (h0 < G) sc[h0 * kChunkCap + rA] = c[0] * a.scale_log2;
-        if (h1 < G) sc[h1 * kChunkCap + rA] = c[1] * a.scale_log2;
+        if (h0 < G) sc[h0 * kScStride + rA] = c[0] * a.scale_log2;
+        if (h1 < G) sc[h1 * kScStride + rA] = c[1] * a.scale_log2;
       }
       if (rB < clen) {
-        if (h0 < G) sc[h0 * kChunkCap + rB] = c[2] * a.scale_log2;
-        if (h1 < G) sc[h1 * kChunkCap + rB] = c[3] * a.scale_log2;
+        if (h0 < G) sc[h0 * kScStride + rB] = c[2] * a.scale_log2;
+        if (h1 < G) sc[h1 * kScStride + rB] = c[3] * a.scale_log2;
       }
     }
   }
@@ -181,7 +176,7 @@ __global__ void __launch_bounds__(kThreads, COWA_DEC_MINB) cowa_decode_split_ker
 
   // ---------------- phase 2: max, exp2, sum per head ----------------
   for (int h = warp; h < G; h += kThreads / 32) {
-    float* s = sc + h * kChunkCap;
+    float* s = sc + h * kScStride;
     float m = -INFINITY;
     for (int r = lane; r < clen; r += 32) m = fmaxf(m, s[r]);
 #pragma unroll
@@ -198,53 +193,67 @@ __global__ void __launch_bounds__(kThreads, COWA_DEC_MINB) cowa_decode_split_ker
   }
   __syncthreads();
 
-  // ---------------- phase 3: values ----------------
-  const int dch = tid % DC, rs = tid / DC;
-  float acc[G][8];
+  // ---------------- phase 3: values, O^T[d, h] += V^T[d, rows] P^T[rows, h] on the tensor cores ----------------
+  // 16 visible rows per mma.  A = V^T: thread (g, t) loads 16 bytes (8 consecutive d) of rows 2t, 2t+1, 2t+8,
+  // 2t+9 and pairs equal d of neighbouring rows with byte permutes; the row index of an m-tile is a
+  // permutation of d (row g <-> d = 8g + 2i, row g+8 <-> d = 8g + 2i + 1 for m-tile i), undone when the
+  // accumulators are written out.  B = P^T (bf16), head g of the group in column g.
+  {
+    const int g = lane >> 2, t = lane & 3;
+    constexpr int NB = D / 64;
+    float acc[NB][4][4];
 #pragma unroll
-  for (int h = 0; h < G; ++h)
+    for (int bb = 0; bb < NB; ++bb)
 #pragma unroll
-    for (int i = 0; i < 8; ++i) acc[h][i] = 0.f;
-
-#ifndef COWA_DEC_U
-#define COWA_DEC_U 4
-#endif
-  constexpr int U = COWA_DEC_U;
-  for (int r0 = rs; r0 < clen; r0 += RP * U) {
-    uint4 vv[U];
+      for (int i = 0; i < 4; ++i)
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int r = min(r0 + u * RP, clen - 1);
-      vv[u] = ldg128(vbase + (size_t)vm.token(c0 + r) * D + dch * 8);
-    }
+        for (int c = 0; c < 4; ++c) acc[bb][i][c] = 0.f;
+    const int nblk = (clen + 15) >> 4;
+    for (int blk = warp; blk < nblk; blk += kThreads / 32) {
+      const int r0 = blk * 16 + 2 * t;
+      const int rr[4] = {r0, r0 + 1, r0 + 8, r0 + 9};
+      uint4 vv[4][NB];
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int r = r0 + u * RP;
-      if (r < clen) {
-        float x[8] = {bf16lo(vv[u].x), bf16hi(vv[u].x), bf16lo(vv[u].y), bf16hi(vv[u].y),
-                      bf16lo(vv[u].z), bf16hi(vv[u].z), bf16lo(vv[u].w), bf16hi(vv[u].w)};
+      for (int k = 0; k < 4; ++k) {
+        const __nv_bfloat16* src = vbase + (size_t)vm.token(c0 + min(rr[k], clen - 1)) * D + g * 8;
 #pragma unroll
-        for (int h = 0; h < G; ++h) {
-          const float p = sc[h * kChunkCap + r];
+        for (int bb = 0; bb < NB; ++bb) vv[k][bb] = ldg128(src + bb * 64);
+      }
+      float pr[4];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) acc[h][i] = fmaf(p, x[i], acc[h][i]);
-        }
+      for (int k = 0; k < 4; ++k) pr[k] = (g < G && rr[k] < clen) ? sc[g * kScStride + rr[k]] : 0.f;
+      uint32_t b0, b1;
+      asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(b0) : "f"(pr[1]), "f"(pr[0]));
+      asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(b1) : "f"(pr[3]), "f"(pr[2]));
+#pragma unroll
+      for (int bb = 0; bb < NB; ++bb) {
+        const uint32_t x0[4] = {vv[0][bb].x, vv[0][bb].y, vv[0][bb].z, vv[0][bb].w};
+        const uint32_t x1[4] = {vv[1][bb].x, vv[1][bb].y, vv[1][bb].z, vv[1][bb].w};
+        const uint32_t x2[4] = {vv[2][bb].x, vv[2][bb].y, vv[2][bb].z, vv[2][bb].w};
+        const uint32_t x3[4] = {vv[3][bb].x, vv[3][bb].y, vv[3][bb].z, vv[3][bb].w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          mma_bf16_16816(acc[bb][i], __byte_perm(x0[i], x1[i], 0x5410), __byte_perm(x0[i], x1[i], 0x7632),
+                         __byte_perm(x2[i], x3[i], 0x5410), __byte_perm(x2[i], x3[i], 0x7632), b0, b1);
       }
     }
-  }
-  __syncthreads();  // scores no longer needed: reuse as red[rs][h][d]  (RP * D == kChunkCap)
-  static_assert(RP * D <= kChunkCap, "reduction buffer fits the score buffer");
+    __syncthreads();  // scores no longer needed: reuse their space as red[warp][h][d]
+    static_assert((kThreads / 32) * D <= kChunkCap, "reduction buffer fits the score buffer");
 #pragma unroll
-  for (int h = 0; h < G; ++h) {
-    float4* dst = reinterpret_cast<float4*>(sc + ((size_t)(rs * G + h) * D + dch * 8));
-    dst[0] = make_float4(acc[h][0], acc[h][1], acc[h][2], acc[h][3]);
-    dst[1] = make_float4(acc[h][4], acc[h][5], acc[h][6], acc[h][7]);
+    for (int bb = 0; bb < NB; ++bb)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int d = bb * 64 + 8 * g + 2 * i;
+        const int h0 = 2 * t, h1 = 2 * t + 1;
+        if (h0 < G) *reinterpret_cast<float2*>(sc + ((size_t)(warp * G + h0) * D + d)) = make_float2(acc[bb][i][0], acc[bb][i][2]);
+        if (h1 < G) *reinterpret_cast<float2*>(sc + ((size_t)(warp * G + h1) * D + d)) = make_float2(acc[bb][i][1], acc[bb][i][3]);
+      }
   }
   __syncthreads();
   for (int i = tid; i < G * D; i += kThreads) {
     float s = 0.f;
 #pragma unroll
-    for (int r = 0; r < RP; ++r) s += sc[r * G * D + i];
+    for (int r = 0; r < kThreads / 32; ++r) s += sc[r * G * D + i];
     a.ws_o[((head0 + i / D) * a.S + split) * D + (i % D)] = s;
   }
   if (tid < G) {
@@ -343,7 +352,7 @@ int max_visible(int Tmax, int hg, const cowa_params_t* p) {
 }
 
 // Blocks of the split kernel that fit the current device at once (SM count x resident blocks per SM).
-// Falls back to 148 x 7 (B200, 72 registers, 16 KB shared memory) when no device can be queried.
+// Falls back to 148 x 5 (B200, up to 102 registers per thread) when no device can be queried.
 template <int D, int G>
 int resident_blocks_of() {
   int dev = 0, sms = 0, occ = 0;
@@ -363,7 +372,7 @@ int resident_blocks(int D, int G) {
                     : G == 4 ? resident_blocks_of<128, 4>() : resident_blocks_of<128, 8>();
     else r = G == 1 ? resident_blocks_of<64, 1>() : G == 2 ? resident_blocks_of<64, 2>()
              : G == 4 ? resident_blocks_of<64, 4>() : resident_blocks_of<64, 8>();
-    if (r <= 0) { cudaGetLastError(); return 148 * 7; }
+    if (r <= 0) { cudaGetLastError(); return 148 * 5; }
     cache[di][gi] = r;
   }
   return cache[di][gi];
