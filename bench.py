@@ -218,8 +218,9 @@ def run_cuda(args):
         cd["B"] = args.decode_batch
     B, T, Hq, Hkv, D = ct["B"], ct["T"], ct["Hq"], ct["Hkv"], ct["D"]
     scale = cowa_inputs.softmax_scale(D)
-    p_train = cowa.make_params(sink=ct["sink"], local=ct["local"], softmax_scale=scale)
-    p_full = cowa.make_params(softmax_scale=scale, full_attn=True)
+    p_train = cowa.make_params(sink=ct["sink"], local=ct["local"], softmax_scale=scale,
+                               deterministic=args.deterministic)
+    p_full = cowa.make_params(softmax_scale=scale, full_attn=True, deterministic=args.deterministic)
     p_dec = cowa.make_params(sink=cd["sink"], local=cd["local"], softmax_scale=scale)
 
     # ---- inputs resident in HBM ----
@@ -421,7 +422,7 @@ def run_cuda(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": args.train_cfg, "decode_workload": DECODE_CFG, "decode_batch": cd["B"], "B": B, "T": T, "Hq": Hq, "Hkv": Hkv,
-                   "D": D, "sink": ct["sink"], "near": ct["local"],
+                   "D": D, "sink": ct["sink"], "near": ct["local"], "deterministic_dq": bool(args.deterministic),
                    "phases": ["fwd"] + (["bwd"] if have_bwd else []) + ["decode"],
                    "l2": "inputs larger than L2 (2.6 GB training tensors, 0.57 GB visible KV cache)",
                    "parallelism": "independent replicas" if world > 1 else "single GPU"},
@@ -452,6 +453,8 @@ def main():
     ap.add_argument("--train-cfg", default=TRAIN_CFG, choices=["8k", "32k", "128k"],
                     help="training configuration (default: the 128K headline; smaller ones are for profiling)")
     ap.add_argument("--decode-batch", type=int, default=0, help="override the decode batch (profiling)")
+    ap.add_argument("--deterministic", action="store_true",
+                    help="backward with fixed-point dQ accumulation (bitwise reproducible dQ)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

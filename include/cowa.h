@@ -64,6 +64,11 @@ typedef struct {
                                    Read during the call; not retained.  Ignored by cowa_decode. */
   int32_t full_attn;   /* 1 => every head sees the whole causal prefix (dense FullAttn path) */
   float softmax_scale; /* scores are softmax_scale * q.k (the paper pre-scales Q by 1/sqrt(d_h)) */
+  int32_t deterministic; /* cowa_bwd only.  0: dQ partial sums are added in fp32 in whatever order the
+                            blocks arrive (Algorithm 2 line 15's AtomicAdd; results vary in the last bits
+                            from run to run).  1: the partial sums are added as 32-bit fixed point with
+                            18 fractional bits, which is exact and order-independent, so dQ is bitwise
+                            reproducible; requires |dQ| < 8192 and rounds each partial to 2^-19. */
 } cowa_params_t;
 
 /* Training / prefill forward, Algorithm 1.  N_q = N_k = T.
@@ -83,7 +88,8 @@ int cowa_prefill(const void* q, const void* k, const void* v, void* o, float* ls
 /* Training backward, Algorithm 2: exact gradient of cowa_fwd.
  *   in: q,k,v,o,lse as produced by cowa_fwd, d_o [B,Hq,T,D];
  *   out: dq [B,Hq,T,D], dk,dv [B,Hkv,T,D] bf16 (fully overwritten).
- * dk,dv are summed over the QO heads of each group inside one thread block (no atomics);
+ * dk,dv are summed over the QO heads of each group inside one thread block (no atomics) and are always
+ * bitwise reproducible; for dq see cowa_params_t.deterministic.
  * `workspace` (device, >= cowa_bwd_workspace_bytes, 16-byte aligned) holds the fp32
  * row vector rowsum(o*d_o) (Algorithm 2 line 13) and needs no initialisation. */
 int cowa_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse,

@@ -30,7 +30,7 @@ class Params(C.Structure):
     _fields_ = [
         ("sink", C.c_int32), ("local", C.c_int32), ("block_q", C.c_int32), ("block_k", C.c_int32),
         ("hkv_global", C.c_int32), ("hkv_offset", C.c_int32), ("windows", C.POINTER(Window)),
-        ("full_attn", C.c_int32), ("softmax_scale", C.c_float),
+        ("full_attn", C.c_int32), ("softmax_scale", C.c_float), ("deterministic", C.c_int32),
     ]
 
 
@@ -81,7 +81,7 @@ def lib():
 
 
 def make_params(sink=0, local=1, block=128, softmax_scale=1.0, windows=None, full_attn=False,
-                hkv_global=0, hkv_offset=0, block_q=None, block_k=None):
+                hkv_global=0, hkv_offset=0, block_q=None, block_k=None, deterministic=False):
     """Fills a cowa_params_t.  `windows`: optional list of (sink, near, gap, len) per KV head."""
     p = Params()
     p.sink, p.local = int(sink), int(local)
@@ -90,6 +90,7 @@ def make_params(sink=0, local=1, block=128, softmax_scale=1.0, windows=None, ful
     p.hkv_global, p.hkv_offset = int(hkv_global), int(hkv_offset)
     p.full_attn = 1 if full_attn else 0
     p.softmax_scale = float(softmax_scale)
+    p.deterministic = 1 if deterministic else 0
     if windows is not None:
         arr = (Window * len(windows))(*[Window(*map(int, w)) for w in windows])
         p.windows = C.cast(arr, C.POINTER(Window))

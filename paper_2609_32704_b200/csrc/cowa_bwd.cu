@@ -39,6 +39,7 @@ namespace {
 constexpr int BKV = 128;  // KV rows per block (MMA M)
 constexpr int BQS = 64;   // QO rows per step (MMA N of S^T / dP^T)
 constexpr int NST = 3;    // Q / dO stages
+constexpr float kDqFixedOne = 262144.f;  // 2^18: one unit of dQ in the fixed-point accumulation mode
 
 struct BwdArgs {
   const float* lse2;   // [B*Hq, Tpad]  LSE * log2(e)
@@ -47,6 +48,7 @@ struct BwdArgs {
   unsigned int* status;
   int B, Nq, Nk, Hq, Hkv, G, Tpad;
   int sink_tiles;      // KV tiles per head that hold sink columns (launched first)
+  int dq_fixed;        // 1: dQ partial sums travel as 32-bit fixed point (order-independent addition)
   float scale, scale_log2;
   CowaHeadWindows wins;
 };
@@ -476,8 +478,15 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           if (issuer) tma_wait_group_read<1>();  // the reduction issued from this tile one step ago has read it
           wg_sync(3);
           if (d < D) {
+            if (a.dq_fixed) {
+              const float fx = a.scale * kDqFixedOne;
 #pragma unroll
-            for (int c = 0; c < 32; ++c) stage[c * D + d] = __uint_as_float(v[hf][c]) * a.scale;
+              for (int c = 0; c < 32; ++c)
+                reinterpret_cast<int*>(stage)[c * D + d] = __float2int_rn(__uint_as_float(v[hf][c]) * fx);
+            } else {
+#pragma unroll
+              for (int c = 0; c < 32; ++c) stage[c * D + d] = __uint_as_float(v[hf][c]) * a.scale;
+            }
           }
           fence_proxy_async_smem();
           wg_sync(3);
@@ -534,7 +543,7 @@ __global__ void cowa_bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, 
 
 template <int D>
 __global__ void cowa_bwd_convert_dq_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dq, int T,
-                                           int Tpad, long long BH) {
+                                           int Tpad, long long BH, int fixed) {
   const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;  // one thread per 8 elements
   const long long total = BH * T * (D / 8);
   if (gid >= total) return;
@@ -543,7 +552,12 @@ __global__ void cowa_bwd_convert_dq_kernel(const float* __restrict__ acc, __nv_b
   const long long bh = row / T;
   const int t = (int)(row % T);
   const float4* src = reinterpret_cast<const float4*>(acc + ((size_t)bh * Tpad + t) * D + part * 8);
-  const float4 x = src[0], y = src[1];
+  float4 x = src[0], y = src[1];
+  if (fixed) {  // the accumulator holds 32-bit integers in units of 2^-18
+    const float u = 1.f / kDqFixedOne;
+    x = make_float4(__float_as_int(x.x) * u, __float_as_int(x.y) * u, __float_as_int(x.z) * u, __float_as_int(x.w) * u);
+    y = make_float4(__float_as_int(y.x) * u, __float_as_int(y.y) * u, __float_as_int(y.z) * u, __float_as_int(y.w) * u);
+  }
   uint4 v;
   v.x = pack_bf16(x.x, x.y); v.y = pack_bf16(x.z, x.w); v.z = pack_bf16(y.x, y.y); v.w = pack_bf16(y.z, y.w);
   *reinterpret_cast<uint4*>(dq + ((size_t)bh * T + t) * D + part * 8) = v;
@@ -575,7 +589,9 @@ int launch_bwd(const void* q, const void* k, const void* v, const void* o, const
   }
   CUtensorMap mq, mk, mv, mdo, mdk, mdv, mdq;
   int rc;
-  if ((rc = cowa::make_tensor_map_3d(&mdq, dq_acc, cowa::MapType::F32, D, Tpad, BH, D, 32, false))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mdq, dq_acc, p->deterministic ? cowa::MapType::S32 : cowa::MapType::F32, D, Tpad, BH, D,
+                                     32, false)))
+    return rc;
   if ((rc = cowa::make_tensor_map_3d(&mq, q, cowa::MapType::BF16, D, T, BH, 64, BQS))) return rc;
   if ((rc = cowa::make_tensor_map_3d(&mdo, d_o, cowa::MapType::BF16, D, T, BH, 64, BQS))) return rc;
   if ((rc = cowa::make_tensor_map_3d(&mk, k, cowa::MapType::BF16, D, T, (long long)B * Hkv, 64, BKV))) return rc;
@@ -591,6 +607,7 @@ int launch_bwd(const void* q, const void* k, const void* v, const void* o, const
   a.scale_log2 = p->softmax_scale * 1.4426950408889634f;
   a.wins = hw;
   a.sink_tiles = 0;
+  a.dq_fixed = p->deterministic ? 1 : 0;
   for (int h = 0; h < Hkv; ++h) {
     const int sk = hw.w[h].s < T ? hw.w[h].s : T;
     a.sink_tiles = std::max(a.sink_tiles, (sk + BKV - 1) / BKV);
@@ -606,7 +623,7 @@ int launch_bwd(const void* q, const void* k, const void* v, const void* o, const
   {
     const long long threads = BH * T * (D / 8);
     cowa_bwd_convert_dq_kernel<D><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(
-        dq_acc, static_cast<__nv_bfloat16*>(dq), T, Tpad, BH);
+        dq_acc, static_cast<__nv_bfloat16*>(dq), T, Tpad, BH, p->deterministic ? 1 : 0);
     COWA_CUDA_TRY(cudaGetLastError());
   }
   return COWA_OK;

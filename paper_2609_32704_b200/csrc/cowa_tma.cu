@@ -30,7 +30,10 @@ int make_tensor_map_3d(CUtensorMap* map, const void* base, MapType type, int D, 
   cuuint64_t strides[2] = {(cuuint64_t)D * es, (cuuint64_t)D * es * (cuuint64_t)T};
   cuuint32_t box[3] = {(cuuint32_t)box_d, (cuuint32_t)box_t, 1};
   cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = fn(map, type == MapType::BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+  const CUtensorMapDataType dt = type == MapType::BF16  ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
+                                 : type == MapType::F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                                        : CU_TENSOR_MAP_DATA_TYPE_INT32;
+  CUresult r = fn(map, dt,
                   3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                   swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);

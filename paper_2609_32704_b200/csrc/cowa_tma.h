@@ -7,7 +7,7 @@
 
 namespace cowa {
 
-enum class MapType { BF16, F32 };
+enum class MapType { BF16, F32, S32 };
 
 // Builds a 3-D map with dims (D, T, BH) and box (box_d, box_t, 1); with `swizzle128` the shared
 // memory side uses the 128-byte swizzle (box_d * element size must then be 128 bytes or less),

@@ -209,6 +209,24 @@ def test_bwd_dkdv_bitwise_repeatable():
     assert torch.equal(dk1, dk2) and torch.equal(dv1, dv2)
 
 
+def test_bwd_deterministic_dq():
+    # Fixed-point accumulation of the dQ partial sums: bitwise equal from run to run, and still within
+    # the parity tolerance.
+    B, T, Hq, Hkv, D, sink, local = 1, 4096, 8, 2, 128, 64, 512
+    q, k, v, d_o = cowa_inputs.make_train_inputs(55, B, T, Hq, Hkv, D)
+    scale = cowa_inputs.softmax_scale(D)
+    params = cowa.make_params(sink=sink, local=local, softmax_scale=scale, deterministic=True)
+    args = [x.to(DEV) for x in (q, k, v, d_o)]
+    dq1, dk1, dv1 = run_fwd_bwd(*args, params)
+    dq2, dk2, dv2 = run_fwd_bwd(*args, params)
+    assert torch.equal(dq1, dq2) and torch.equal(dk1, dk2) and torch.equal(dv1, dv2)
+    ws = orc.default_windows(T, Hkv, sink, local)
+    f = cowa_inputs.to_f64
+    for h in (0, 5):
+        ref = orc.backward_dq_rows(f(q[0]), f(k[0]), f(v[0]), f(d_o[0]), ws, scale, h, np.arange(T))
+        check_grad(f"deterministic dq[{h}]", dq1[0, h].float().cpu().numpy(), ref)
+
+
 def test_bwd_8k_config_sampled():
     c = cowa_inputs.CONFIGS["8k"]
     B, T, Hq, Hkv, D = c["B"], c["T"], c["Hq"], c["Hkv"], c["D"]
