@@ -17,6 +17,7 @@ operator has no exchange step); rank 0 prints one JSON line.
 from __future__ import annotations
 
 import argparse
+import itertools
 import json
 import os
 import statistics
@@ -352,6 +353,54 @@ def run_cuda(args):
                      "byte_ratio_decode": sum(lens_h) * cd["Hkv"] / vis_rows})
         del ws_df
 
+    # ---- prefill over a packed batch of mixed lengths (one launch) against one call per sequence ----
+    varlen = None
+    if not args.no_varlen:
+        mix = [65536, 32768, 16384, 16384, 8192, 8192, 4096, 2048, 1000, 333]  # N_q = N_k per sequence
+        tot = sum(mix)
+        pq, pk, pv, _ = cowa_inputs.make_train_inputs(7, 1, tot, Hq, Hkv, D, device=dev)
+        pq, pk, pv = pq[0], pk[0], pv[0]
+        po = torch.empty_like(pq)
+        plse = torch.empty((Hq, tot), dtype=torch.float32, device=dev)
+        cu = torch.tensor([0] + list(itertools.accumulate(mix)), dtype=torch.int32, device=dev)
+        p_mix = cowa.make_params(sink=ct["sink"], local=ct["local"], softmax_scale=scale)
+        v_flops = sum(cowa.cowa_tile_counts(n, n, Hkv, p_mix)["visited"] for n in mix) * 128 * 128 * 4 * D * G
+
+        def packed():
+            cowa.cowa_prefill_varlen(pq, pk, pv, po, plse, cu, cu, p_mix)
+
+        def one_by_one():
+            a0 = 0
+            for n in mix:
+                # a sequence's rows are not contiguous per head inside the packed tensors: time on copies
+                cowa.cowa_prefill(seq_q[a0], seq_k[a0], seq_v[a0], seq_o[a0], seq_l[a0], p_mix)
+                a0 += n
+
+        seq_q, seq_k, seq_v, seq_o, seq_l = {}, {}, {}, {}, {}
+        a0 = 0
+        for n in mix:
+            seq_q[a0] = pq[:, a0:a0 + n].contiguous()[None]
+            seq_k[a0] = pk[:, a0:a0 + n].contiguous()[None]
+            seq_v[a0] = pv[:, a0:a0 + n].contiguous()[None]
+            seq_o[a0] = torch.empty_like(seq_q[a0])
+            seq_l[a0] = torch.empty((1, Hq, n), dtype=torch.float32, device=dev)
+            a0 += n
+        times = {}
+        for name, fn in (("packed", packed), ("one_by_one", one_by_one)):
+            for _ in range(2):
+                fn()
+            ev2 = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+            ev2[0].record()
+            for _ in range(5):
+                fn()
+            ev2[1].record()
+            torch.cuda.synchronize()
+            times[name] = max_over_ranks(ev2[0].elapsed_time(ev2[1]) / 5, world)
+        cowa.cowa_check_device_status()
+        varlen = {"lengths": mix, "ms": times["packed"], "tflops": v_flops / times["packed"] / 1e9,
+                  "one_call_per_sequence_ms": times["one_by_one"]}
+        del pq, pk, pv, po, plse, seq_q, seq_k, seq_v, seq_o, seq_l
+
     # ---- end to end: host buffers in, results back to the host, copies inside the timed region ----
     e2e = None
     if not args.no_e2e:
@@ -453,7 +502,7 @@ def run_cuda(args):
         "bwd_ms": bwd_ms if have_bwd else None, "bwd_tflops": bwd_flops / bwd_ms / 1e9 if have_bwd else None,
         "bwd_main_kernel_ms": bwd_main_ms,
         "visited_tiles": cnt["visited"], "causal_tiles": cnt["causal"],
-        "decode": decode, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
+        "decode": decode, "prefill_varlen": varlen, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
         "gpu_launches": args.steps * (1 + (BWD_LAUNCHES if have_bwd else 0) + 2),
     }
     line.update(full)
@@ -471,6 +520,7 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-fullattn", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-varlen", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--train-cfg", default=TRAIN_CFG, choices=["8k", "32k", "128k"],

@@ -44,7 +44,9 @@ typedef enum {
   COWA_ERR_WORKSPACE_TOO_SMALL = -4,
   COWA_ERR_CUDA = -5,               /* a CUDA call failed; see cowa_last_cuda_error() */
   COWA_ERR_DEVICE_TIMEOUT = -6,     /* reported by cowa_check_device_status(): a bounded device wait ran out */
-  COWA_ERR_STATIC_SCRATCH_EXCEEDED = -7 /* cowa_decode_static: the call needs more scratch than the built-in array holds */
+  COWA_ERR_STATIC_SCRATCH_EXCEEDED = -7, /* cowa_decode_static: the call needs more scratch than the built-in array holds */
+  COWA_ERR_DEVICE_BAD_SEQLENS = -8  /* reported by cowa_check_device_status(): cowa_prefill_varlen met a sequence
+                                       with N_q > N_k in its device-side offset arrays and skipped it */
 } cowa_status_t;
 
 /* One KV head's windows: the paper's 4-tuple (sink width, near width, gap after the
@@ -84,6 +86,23 @@ int cowa_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
  * Every sequence of the batch has the same Nq and Nk.  cowa_fwd is this call with Nq = Nk = T. */
 int cowa_prefill(const void* q, const void* k, const void* v, void* o, float* lse,
                  int B, int Nq, int Nk, int Hq, int Hkv, int D, const cowa_params_t* p, void* stream);
+
+/* Prefill over a packed batch of B sequences of different lengths (Sec. 2.1: each sequence b has its own
+ * N_q[b] <= N_k[b]; its queries sit at key positions i_q + (N_k[b] - N_q[b]), Eq. fwa_distance, and its
+ * long-range breakpoints follow from its own N_k[b], Eq. fwa_long_range_span; Sec. 2.3 "Forward execution").
+ *   q [Hq,total_q,D]; k,v [Hkv,total_k,D] in; o [Hq,total_q,D] bf16 and lse [Hq,total_q] fp32 out: the
+ *   sequences are concatenated along the token axis, head-major, contiguous.
+ *   cu_seqlens_q, cu_seqlens_k: DEVICE int32[B+1], non-decreasing row offsets with cu[0] = 0,
+ *   cu_q[B] = total_q, cu_k[B] = total_k; sequence b owns rows [cu[b], cu[b+1]).  N_q[b] = 0 is allowed
+ *   (the sequence is skipped).
+ * Explicit tuples in p->windows apply to every sequence unchanged; the default rule and full_attn are
+ * evaluated per sequence on the device.  The offsets are read on the device only: a sequence with
+ * N_q > N_k, or whose rows leave the tensors, is skipped (N_q < 0 counts as empty) and
+ * cowa_check_device_status() then returns COWA_ERR_DEVICE_BAD_SEQLENS.  No workspace; nothing is
+ * retained.  Blocks are issued sequence after sequence: passing long sequences first shortens the tail. */
+int cowa_prefill_varlen(const void* q, const void* k, const void* v, void* o, float* lse,
+                        const int32_t* cu_seqlens_q, const int32_t* cu_seqlens_k, int B, int total_q,
+                        int total_k, int Hq, int Hkv, int D, const cowa_params_t* p, void* stream);
 
 /* Training backward, Algorithm 2: exact gradient of cowa_fwd.
  *   in: q,k,v,o,lse as produced by cowa_fwd, d_o [B,Hq,T,D];
@@ -171,7 +190,8 @@ int cowa_tile_counts(int Nq, int Nk, int Hkv, const cowa_params_t* p, int64_t ou
 
 /* The kernels bound every device-side wait; a wait that runs out sets a flag in a device word
  * instead of hanging.  This call synchronises `stream`, reads and clears the flag, and returns
- * COWA_OK or COWA_ERR_DEVICE_TIMEOUT (COWA_ERR_CUDA if the stream itself reports an error). */
+ * COWA_OK, COWA_ERR_DEVICE_TIMEOUT or COWA_ERR_DEVICE_BAD_SEQLENS (COWA_ERR_CUDA if the stream itself
+ * reports an error). */
 int cowa_check_device_status(void* stream);
 
 const char* cowa_status_string(int status);

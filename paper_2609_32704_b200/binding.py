@@ -50,6 +50,8 @@ def lib():
         L.cowa_fwd.restype = i32
         L.cowa_prefill.argtypes = [vp] * 5 + [i32] * 6 + [pp, vp]
         L.cowa_prefill.restype = i32
+        L.cowa_prefill_varlen.argtypes = [vp] * 7 + [i32] * 6 + [pp, vp]
+        L.cowa_prefill_varlen.restype = i32
         L.cowa_bwd.argtypes = [vp] * 9 + [i32] * 5 + [pp, vp, sz, vp]
         L.cowa_bwd.restype = i32
         L.cowa_decode.argtypes = [vp] * 6 + [i32] * 5 + [pp, vp, sz, vp]
@@ -140,6 +142,25 @@ def cowa_prefill(q, k, v, o, lse, params):
     Hkv, Nk = k.shape[1], k.shape[2]
     _check(lib().cowa_prefill(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), B, Nq, Nk, Hq, Hkv, D,
                               C.byref(params), _stream()), "cowa_prefill")
+
+
+def cowa_prefill_varlen(q, k, v, o, lse, cu_seqlens_q, cu_seqlens_k, params):
+    """Packed batch: q [Hq,total_q,D], k/v [Hkv,total_k,D] -> o, lse [Hq,total_q]; cu_seqlens_* are CUDA int32
+    tensors of B+1 row offsets."""
+    import torch
+    for t, n in ((q, "q"), (k, "k"), (v, "v"), (o, "o")):
+        _need(t, torch.bfloat16, n)
+    _need(lse, torch.float32, "lse")
+    _need(cu_seqlens_q, torch.int32, "cu_seqlens_q")
+    _need(cu_seqlens_k, torch.int32, "cu_seqlens_k")
+    if cu_seqlens_q.numel() != cu_seqlens_k.numel() or cu_seqlens_q.numel() < 2:
+        raise ValueError("cu_seqlens_q and cu_seqlens_k must both hold B+1 offsets")
+    Hq, total_q, D = q.shape
+    Hkv, total_k = k.shape[0], k.shape[1]
+    B = cu_seqlens_q.numel() - 1
+    _check(lib().cowa_prefill_varlen(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(cu_seqlens_q),
+                                     _ptr(cu_seqlens_k), B, total_q, total_k, Hq, Hkv, D,
+                                     C.byref(params), _stream()), "cowa_prefill_varlen")
 
 
 def cowa_bwd_workspace_bytes(B, T, Hq, Hkv, D, params):

@@ -167,7 +167,7 @@ int cowa_check_device_status(void* stream) {
   if (host != 0) {
     COWA_CUDA_TRY(cudaMemsetAsync(word, 0, sizeof(host), s));
     COWA_CUDA_TRY(cudaStreamSynchronize(s));
-    return COWA_ERR_DEVICE_TIMEOUT;
+    return (host & 1u) ? COWA_ERR_DEVICE_TIMEOUT : COWA_ERR_DEVICE_BAD_SEQLENS;
   }
   return COWA_OK;
 }
@@ -183,6 +183,8 @@ const char* cowa_status_string(int status) {
     case COWA_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
     case COWA_ERR_STATIC_SCRATCH_EXCEEDED:
       return "cowa_decode_static: the call needs more scratch than the library's built-in array holds";
+    case COWA_ERR_DEVICE_BAD_SEQLENS:
+      return "cowa_prefill_varlen: a sequence with N_q > N_k was skipped";
     default: return "unknown status";
   }
 }

@@ -30,9 +30,15 @@ constexpr int kFwdThreads = 160;
 struct FwdArgs {
   float* lse;
   unsigned int* status;
-  int B, Nq, Nk, Hq, Hkv, G;
+  int B, Nq, Nk, Hq, Hkv, G;  // packed batches: Nq, Nk unused
   float scale_log2;
   CowaHeadWindows wins;
+  // packed (variable-length) batches only
+  const int* cu_q;   // [B+1] row offsets of the sequences in q / o / lse
+  const int* cu_k;   // [B+1] row offsets in k / v
+  __nv_bfloat16* o;  // raw output pointer for the last, partial tile of a sequence
+  int total_q, total_k;
+  int sink, local, hkv_global, hkv_offset, full_attn, explicit_windows;
 };
 
 // bits [lo, hi] of the 32-bit word covering columns [base, base+32)
@@ -50,7 +56,7 @@ struct FwdSmem {
   static constexpr int kBytes = oBar + 128 + 1024;  // + barriers + alignment slack
 };
 
-template <int D>
+template <int D, bool VARLEN>
 __global__ void __launch_bounds__(kFwdThreads, 2)
 cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
@@ -85,17 +91,63 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   int idx = blockIdx.x;
   const int g = idx % a.G; idx /= a.G;
   const int hk = idx % a.Hkv; idx /= a.Hkv;
-  const int b = idx % a.B; idx /= a.B;
-  const int nQ = (a.Nq + BQ - 1) / BQ;
-  const int i = nQ - 1 - idx;
+  int b, i;
+  if constexpr (!VARLEN) {
+    b = idx % a.B; idx /= a.B;
+    i = (a.Nq + BQ - 1) / BQ - 1 - idx;
+  } else {
+    // idx counts the QO tiles of the packed batch, sequence after sequence, each sequence's heaviest
+    // (last) tile first.  Every warp finds its (sequence, tile) by a cooperative scan of the offsets.
+    const int lane = threadIdx.x & 31;
+    int base = 0;
+    b = -1; i = 0;
+    for (int b0 = 0; b0 < a.B; b0 += 32) {
+      const int bb = b0 + lane;
+      const int n = bb < a.B ? a.cu_q[bb + 1] - a.cu_q[bb] : 0;
+      const int tiles = n > 0 ? (n + BQ - 1) / BQ : 0;
+      int incl = tiles;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += y;
+      }
+      const int tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
+      if (idx < base + tot) {
+        const unsigned m = __ballot_sync(0xFFFFFFFFu, idx < base + incl);
+        const int src = __ffs(m) - 1;
+        const int excl = __shfl_sync(0xFFFFFFFFu, incl - tiles, src);
+        const int nt_seq = __shfl_sync(0xFFFFFFFFu, tiles, src);
+        b = b0 + src;
+        i = nt_seq - 1 - (idx - base - excl);
+        break;
+      }
+      base += tot;
+    }
+    if (b < 0) return;  // the grid is sized from an upper bound of the tile count
+  }
   const int h = hk * a.G + g;
-  const int off = a.Nk - a.Nq;
-  const int q0 = i * BQ, q1 = min(q0 + BQ, a.Nq) - 1;
-  const CowaWin w = a.wins.w[hk];
+  // Sequence geometry.  Packed batches: every sequence has its own N_q <= N_k, its rows start at
+  // cu_q[b] / cu_k[b] of a [H, total, D] tensor, and its windows follow from its own N_k.
+  int Nq = a.Nq, Nk = a.Nk, qbase = 0, kbase = 0;
+  int bhq = b * a.Hq + h, bhk = b * a.Hkv + hk;
+  CowaWin w = a.wins.w[hk];
+  if constexpr (VARLEN) {
+    qbase = a.cu_q[b]; Nq = a.cu_q[b + 1] - qbase;
+    kbase = a.cu_k[b]; Nk = a.cu_k[b + 1] - kbase;
+    bhq = h; bhk = hk;
+    if (Nq > Nk || qbase < 0 || kbase < 0 || qbase + Nq > a.total_q || kbase + Nk > a.total_k) {
+      // malformed offsets: report, touch nothing
+      if (threadIdx.x == 0) atomicOr(a.status, 2u);
+      return;
+    }
+    if (a.full_attn) { w.s = 0; w.n = Nk; w.g = 0; w.l = 0; }
+    else if (!a.explicit_windows) w = cowa_default_window(Nk, a.hkv_global, a.hkv_offset + hk, a.sink, a.local);
+  }
+  const int off = Nk - Nq;
+  const int q0 = i * BQ, q1 = min(q0 + BQ, Nq) - 1;
   CowaRange rg[3];
-  cowa_fwd_ranges(w, q0, q1, off, a.Nk, BK, rg);
+  cowa_fwd_ranges(w, q0, q1, off, Nk, BK, rg);
   const int nt = cowa_range_len(rg[0]) + cowa_range_len(rg[1]) + cowa_range_len(rg[2]);
-  const int bhq = b * a.Hq + h, bhk = b * a.Hkv + hk;
 
   // ---- set-up ----
   if (tid == 0) {
@@ -134,7 +186,7 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           const int j = cowa_fwd_tile_at(rg, t);
           uint8_t* dst = sK + (t & 1) * SM::kKV;
           mbar_expect_tx(bar_k + (t & 1), SM::kKV);
-          for (int s = 0; s < NSLAB; ++s) tma_load_3d(dst + s * SLAB_K, &tmK, bar_k + (t & 1), s * 64, j * BK, bhk);
+          for (int s = 0; s < NSLAB; ++s) tma_load_3d(dst + s * SLAB_K, &tmK, bar_k + (t & 1), s * 64, kbase + j * BK, bhk);
         }
       };
       auto load_v = [&](int t) {
@@ -142,7 +194,7 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           const int j = cowa_fwd_tile_at(rg, t);
           uint8_t* dst = sV + (t & 1) * SM::kKV;
           mbar_expect_tx(bar_v + (t & 1), SM::kKV);
-          for (int s = 0; s < NSLAB; ++s) tma_load_3d(dst + s * SLAB_K, &tmV, bar_v + (t & 1), s * 64, j * BK, bhk);
+          for (int s = 0; s < NSLAB; ++s) tma_load_3d(dst + s * SLAB_K, &tmV, bar_v + (t & 1), s * 64, kbase + j * BK, bhk);
         }
       };
       auto issue_s = [&](int buf) {  // S = Q K^T into TMEM buffer buf from K buffer buf
@@ -158,7 +210,7 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       if (lead) {
         prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV);
         mbar_expect_tx(bar_q, SM::kQ);
-        for (int s = 0; s < NSLAB; ++s) tma_load_3d(sQ + s * SLAB_Q, &tmQ, bar_q, s * 64, q0, bhq);
+        for (int s = 0; s < NSLAB; ++s) tma_load_3d(sQ + s * SLAB_Q, &tmQ, bar_q, s * 64, qbase + q0, bhq);
       }
       load_k(0);
       if (nt > 1) load_k(1);
@@ -202,7 +254,10 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);  // this warp's 32 lanes
     const uint32_t t_O = t_lane + cO;
     const int row = q0 + tid;
-    const bool row_valid = row < a.Nq;
+    const bool row_valid = row < Nq;
+    // Last, partial tile of a packed sequence: the rows after it belong to the next sequence, so the
+    // tile is written row by row instead of by one bulk store.
+    const bool tail_rows = VARLEN && (q0 + BQ > Nq);
     const int rowpos = row + off;  // position of this query on the key axis
     float m_ref = -INFINITY, l_sum = 0.f;
     const float2 sc2 = make_float2(a.scale_log2, a.scale_log2);
@@ -211,7 +266,7 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const int b_ = t & 1;
       const int j = cowa_fwd_tile_at(rg, t);
       const int k0 = j * BK;
-      const bool full = cowa_tile_full(w, q0, BQ, k0, BK, off, a.Nq, a.Nk);
+      const bool full = cowa_tile_full(w, q0, BQ, k0, BK, off, Nq, Nk);
       const uint32_t t_S = t_lane + b_ * 64;
 
       ok = mbar_wait(bar_s + b_, (t >> 1) & 1, a.status);
@@ -223,7 +278,7 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       tmem_wait_ld();
 
       if (!full) {
-        const int kend = min(rowpos, a.Nk - 1);  // last causal key of this row
+        const int kend = min(rowpos, Nk - 1);  // last causal key of this row
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
           const int base = k0 + c * 32;
@@ -315,16 +370,21 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           v.w = pack_bf16(__uint_as_float(ov[q * 8 + 6]) * inv, __uint_as_float(ov[q * 8 + 7]) * inv);
           const int d0 = c * 32 + q * 8;
           const int slab = d0 / 64, chunk = (d0 % 64) / 8;
-          *reinterpret_cast<uint4*>(sQ + slab * SLAB_Q + tid * 128 + ((chunk ^ (tid & 7)) << 4)) = v;
+          if (!tail_rows)
+            *reinterpret_cast<uint4*>(sQ + slab * SLAB_Q + tid * 128 + ((chunk ^ (tid & 7)) << 4)) = v;
+          else if (row_valid)
+            *reinterpret_cast<uint4*>(a.o + ((size_t)h * a.total_q + qbase + row) * D + d0) = v;
         }
       }
-      if (row_valid)
-        a.lse[(size_t)bhq * a.Nq + row] = 0.6931471805599453f * (m_ref + log2f(l_sum));
+      if (row_valid) {
+        const size_t li = VARLEN ? (size_t)h * a.total_q + qbase + row : (size_t)bhq * Nq + row;
+        a.lse[li] = 0.6931471805599453f * (m_ref + log2f(l_sum));
+      }
       fence_proxy_async_smem();
     }
     asm volatile("bar.sync 1, 128;" ::: "memory");  // the four softmax warps
-    if (tid == 0 && ok && nt > 0) {
-      for (int s = 0; s < NSLAB; ++s) tma_store_3d(&tmO, sQ + s * SLAB_Q, s * 64, q0, bhq);
+    if (tid == 0 && ok && nt > 0 && !tail_rows) {
+      for (int s = 0; s < NSLAB; ++s) tma_store_3d(&tmO, sQ + s * SLAB_Q, s * 64, qbase + q0, bhq);
       tma_commit_group();
       tma_wait_group<0>();
     }
@@ -339,15 +399,20 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   }
 }
 
-template <int D>
+// One launch for both layouts.  Batched: cu_q == nullptr, tensors [B,H,N,D].  Packed: tensors
+// [H,total,D]; the grid is sized from total_q / BQ + B, an upper bound of the batch's tile count.
+template <int D, bool VARLEN>
 int launch_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Nq, int Nk, int Hq,
-               int Hkv, const cowa_params_t* p, const CowaHeadWindows& hw, cudaStream_t st) {
+               int Hkv, const cowa_params_t* p, const CowaHeadWindows& hw, const int* cu_q, const int* cu_k,
+               int total_q, int total_k, cudaStream_t st) {
   CUtensorMap mq, mk, mv, mo;
   int rc;
-  if ((rc = cowa::make_tensor_map_3d(&mq, q, cowa::MapType::BF16, D, Nq, (long long)B * Hq, 64, BQ))) return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mk, k, cowa::MapType::BF16, D, Nk, (long long)B * Hkv, 64, BK))) return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mv, v, cowa::MapType::BF16, D, Nk, (long long)B * Hkv, 64, BK))) return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mo, o, cowa::MapType::BF16, D, Nq, (long long)B * Hq, 64, BQ))) return rc;
+  const int rows_q = VARLEN ? total_q : Nq, rows_k = VARLEN ? total_k : Nk;
+  const long long nq_maps = VARLEN ? Hq : (long long)B * Hq, nk_maps = VARLEN ? Hkv : (long long)B * Hkv;
+  if ((rc = cowa::make_tensor_map_3d(&mq, q, cowa::MapType::BF16, D, rows_q, nq_maps, 64, BQ))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mk, k, cowa::MapType::BF16, D, rows_k, nk_maps, 64, BK))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mv, v, cowa::MapType::BF16, D, rows_k, nk_maps, 64, BK))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mo, o, cowa::MapType::BF16, D, rows_q, nq_maps, 64, BQ))) return rc;
   FwdArgs a;
   a.lse = lse;
   a.status = cowa::device_status_word();
@@ -355,11 +420,15 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
   a.B = B; a.Nq = Nq; a.Nk = Nk; a.Hq = Hq; a.Hkv = Hkv; a.G = Hq / Hkv;
   a.scale_log2 = p->softmax_scale * 1.4426950408889634f;
   a.wins = hw;
-  COWA_CUDA_TRY(cudaFuncSetAttribute(cowa_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  a.cu_q = cu_q; a.cu_k = cu_k; a.o = static_cast<__nv_bfloat16*>(o); a.total_q = total_q; a.total_k = total_k;
+  a.sink = p->sink; a.local = p->local;
+  a.hkv_global = p->hkv_global > 0 ? p->hkv_global : Hkv;
+  a.hkv_offset = p->hkv_offset; a.full_attn = p->full_attn; a.explicit_windows = p->windows != nullptr;
+  COWA_CUDA_TRY(cudaFuncSetAttribute(cowa_fwd_kernel<D, VARLEN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      FwdSmem<D>::kBytes));
-  const long long nblocks = (long long)((Nq + BQ - 1) / BQ) * B * Hq;
+  const long long nblocks = VARLEN ? ((long long)total_q / BQ + B) * Hq : (long long)((Nq + BQ - 1) / BQ) * B * Hq;
   if (nblocks > 0x7FFFFFFFll) return COWA_ERR_UNSUPPORTED;
-  cowa_fwd_kernel<D><<<(unsigned)nblocks, kFwdThreads, FwdSmem<D>::kBytes, st>>>(mq, mk, mv, mo, a);
+  cowa_fwd_kernel<D, VARLEN><<<(unsigned)nblocks, kFwdThreads, FwdSmem<D>::kBytes, st>>>(mq, mk, mv, mo, a);
   COWA_CUDA_TRY(cudaGetLastError());
   return COWA_OK;
 }
@@ -380,8 +449,30 @@ int cowa_prefill(const void* q, const void* k, const void* v, void* o, float* ls
   int rc = cowa::resolve_windows(Nk, Hkv, p, &hw);
   if (rc != COWA_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  return D == 128 ? launch_fwd<128>(q, k, v, o, lse, B, Nq, Nk, Hq, Hkv, p, hw, st)
-                  : launch_fwd<64>(q, k, v, o, lse, B, Nq, Nk, Hq, Hkv, p, hw, st);
+  return D == 128 ? launch_fwd<128, false>(q, k, v, o, lse, B, Nq, Nk, Hq, Hkv, p, hw, nullptr, nullptr, 0, 0, st)
+                  : launch_fwd<64, false>(q, k, v, o, lse, B, Nq, Nk, Hq, Hkv, p, hw, nullptr, nullptr, 0, 0, st);
+}
+
+int cowa_prefill_varlen(const void* q, const void* k, const void* v, void* o, float* lse, const int32_t* cu_seqlens_q,
+                        const int32_t* cu_seqlens_k, int B, int total_q, int total_k, int Hq, int Hkv, int D,
+                        const cowa_params_t* p, void* stream) {
+  if (!q || !k || !v || !o || !lse || !p || !cu_seqlens_q || !cu_seqlens_k) return COWA_ERR_INVALID_ARG;
+  if (B <= 0 || total_q <= 0 || total_k < total_q || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0)
+    return COWA_ERR_INVALID_ARG;
+  if (!(p->softmax_scale > 0.f)) return COWA_ERR_INVALID_ARG;
+  if (D != 64 && D != 128) return COWA_ERR_UNSUPPORTED;
+  if (!cowa::aligned16(q) || !cowa::aligned16(k) || !cowa::aligned16(v) || !cowa::aligned16(o))
+    return COWA_ERR_MISALIGNED;
+  // Explicit tuples are validated and copied here; the default rule is evaluated per sequence on the
+  // device (any positive N_k passes the same checks on sink / local / head offsets).
+  CowaHeadWindows hw;
+  int rc = cowa::resolve_windows(total_k, Hkv, p, &hw);
+  if (rc != COWA_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  return D == 128 ? launch_fwd<128, true>(q, k, v, o, lse, B, 0, 0, Hq, Hkv, p, hw, cu_seqlens_q,
+                                          cu_seqlens_k, total_q, total_k, st)
+                  : launch_fwd<64, true>(q, k, v, o, lse, B, 0, 0, Hq, Hkv, p, hw, cu_seqlens_q,
+                                         cu_seqlens_k, total_q, total_k, st);
 }
 
 int cowa_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int T, int Hq, int Hkv, int D,

@@ -141,6 +141,101 @@ def test_prefill_shapes(B, Nq, Nk, Hq, Hkv, D, sink, local):
         check(f"prefill o[b={b}]", o[b].float().cpu().numpy(), o_ref)
 
 
+# ------------------------------------------------------------------ prefill over a packed batch
+
+def _packed_inputs(seed, seqs, Hq, Hkv, D):
+    """Per-sequence inputs concatenated along the token axis: q [Hq,total_q,D], k, v [Hkv,total_k,D]."""
+    qs, ks, vs = [], [], []
+    for b, (nq, nk) in enumerate(seqs):
+        if nq > 0:
+            qs.append(cowa_inputs.make_train_inputs(seed + 2 * b, 1, nq, Hq, Hkv, D)[0][0])
+        _, kb, vb, _ = cowa_inputs.make_train_inputs(seed + 2 * b + 1, 1, nk, Hq, Hkv, D)
+        ks.append(kb[0]); vs.append(vb[0])
+    cu_q = np.concatenate([[0], np.cumsum([s[0] for s in seqs])]).astype(np.int32)
+    cu_k = np.concatenate([[0], np.cumsum([s[1] for s in seqs])]).astype(np.int32)
+    return torch.cat(qs, 1).contiguous(), torch.cat(ks, 1).contiguous(), torch.cat(vs, 1).contiguous(), cu_q, cu_k
+
+
+def _run_varlen(q, k, v, cu_q, cu_k, params):
+    Hq, total_q, _ = q.shape
+    o = torch.full_like(q, float("nan")).to(DEV)
+    lse = torch.full((Hq, total_q), float("nan"), dtype=torch.float32, device=DEV)
+    cowa.cowa_prefill_varlen(q.to(DEV), k.to(DEV), v.to(DEV), o, lse, torch.from_numpy(cu_q).to(DEV),
+                             torch.from_numpy(cu_k).to(DEV), params)
+    torch.cuda.synchronize()
+    return o, lse
+
+
+@pytest.mark.parametrize("seqs,Hq,Hkv,D,sink,local,mode", [
+    ([(100, 100), (1, 700), (300, 1000), (0, 50), (257, 300), (128, 128), (129, 4000)], 4, 2, 128, 16, 100, "default"),
+    ([(64, 64), (65, 129), (1000, 1000), (5, 5)], 8, 2, 64, 5, 60, "default"),
+    ([(200, 900), (333, 333), (1, 1)], 4, 4, 128, 8, 50, "full"),
+    ([(384, 2000), (500, 2000), (77, 1500)], 4, 2, 128, 0, 0, "explicit"),
+])
+def test_prefill_varlen(seqs, Hq, Hkv, D, sink, local, mode):
+    q, k, v, cu_q, cu_k = _packed_inputs(71, seqs, Hq, Hkv, D)
+    scale = cowa_inputs.softmax_scale(D)
+    tuples = None
+    if mode == "explicit":  # the same tuples for every sequence, whatever its length
+        tuples = [(24, 90, 100, 400), (3, 130, 700, 900)][:Hkv]
+        params = cowa.make_params(windows=tuples, softmax_scale=scale)
+    else:
+        params = cowa.make_params(sink=sink, local=local, softmax_scale=scale, full_attn=(mode == "full"))
+    o, lse = _run_varlen(q, k, v, cu_q, cu_k, params)
+    cowa.cowa_check_device_status()
+    f = cowa_inputs.to_f64
+    for b, (nq, nk) in enumerate(seqs):
+        if nq == 0:
+            continue
+        if mode == "explicit":
+            ws = np.array(tuples, dtype=np.int64)
+        elif mode == "full":
+            ws = np.array([(0, nk, 0, 0)] * Hkv, dtype=np.int64)
+        else:
+            ws = orc.default_windows(nk, Hkv, sink, local)
+        qs, ks = slice(cu_q[b], cu_q[b + 1]), slice(cu_k[b], cu_k[b + 1])
+        o_ref, lse_ref = orc.forward(f(q[:, qs]), f(k[:, ks]), f(v[:, ks]), ws, scale)
+        check(f"varlen lse[seq {b}]", lse[:, qs].cpu().numpy(), lse_ref, TOL_LSE, TOL_LSE)
+        check(f"varlen o[seq {b}]", o[:, qs].float().cpu().numpy(), o_ref)
+
+
+def test_prefill_varlen_equals_batched():
+    """Equal-length sequences: the packed call must reproduce the batched call bit for bit."""
+    B, Nq, Nk, Hq, Hkv, D = 3, 384, 1024, 4, 2, 128
+    q, _, _, _ = cowa_inputs.make_train_inputs(81, B, Nq, Hq, Hkv, D)
+    _, k, v, _ = cowa_inputs.make_train_inputs(82, B, Nk, Hq, Hkv, D)
+    params = cowa.make_params(sink=16, local=128, softmax_scale=cowa_inputs.softmax_scale(D))
+    o = torch.empty_like(q).to(DEV)
+    lse = torch.empty((B, Hq, Nq), dtype=torch.float32, device=DEV)
+    cowa.cowa_prefill(q.to(DEV), k.to(DEV), v.to(DEV), o, lse, params)
+    pack = lambda x: x.permute(1, 0, 2, 3).reshape(x.shape[1], -1, x.shape[3]).contiguous()
+    cu_q = (np.arange(B + 1) * Nq).astype(np.int32)
+    cu_k = (np.arange(B + 1) * Nk).astype(np.int32)
+    o2, lse2 = _run_varlen(pack(q), pack(k), pack(v), cu_q, cu_k, params)
+    cowa.cowa_check_device_status()
+    assert torch.equal(pack(o), o2)
+    assert torch.equal(lse.permute(1, 0, 2).reshape(Hq, -1), lse2)
+
+
+def test_prefill_varlen_bad_offsets_reported():
+    """A sequence with N_q > N_k is skipped on the device and reported by the status call; the library
+    stays usable."""
+    seqs = [(64, 64), (100, 200)]
+    q, k, v, cu_q, cu_k = _packed_inputs(91, seqs, 2, 1, 64)
+    params = cowa.make_params(sink=4, local=16, softmax_scale=0.125)
+    bad_q = np.array([0, 24, 164], dtype=np.int32)   # second sequence: 140 queries for ...
+    bad_k = np.array([0, 164, 264], dtype=np.int32)  # ... 100 keys
+    o, _ = _run_varlen(q, k, v, bad_q, bad_k, params)
+    with pytest.raises(cowa.CowaError) as e:
+        cowa.cowa_check_device_status()
+    assert e.value.status == -8
+    assert torch.isnan(o[:, 24:].float()).all()      # nothing of the malformed sequence was written
+    cowa.cowa_check_device_status()                   # flag cleared
+    o, lse = _run_varlen(q, k, v, cu_q, cu_k, params)
+    cowa.cowa_check_device_status()
+    assert torch.isfinite(o.float()).all() and torch.isfinite(lse).all()
+
+
 # ------------------------------------------------------------------ backward
 
 def run_fwd_bwd(q, k, v, d_o, params):
