@@ -509,6 +509,100 @@ def run_cuda(args):
     print(json.dumps(line))
 
 
+# ------------------------------------------------------------------------------------------
+# The paper's operator benchmark re-staged: TP=8 shards of Hq=64, Hkv=8, D=128, batch 1
+# ------------------------------------------------------------------------------------------
+
+# Latency table of the paper (8 x H100, TP=8), ms: T -> (FullAttn fwd, CoWA fwd, FullAttn bwd, CoWA bwd,
+# FullAttn decode, CoWA decode).  Context for the reader, never a target.
+PAPER_TP8_MS = {
+    1024: (0.015, 0.015, 0.055, 0.041, 0.003, 0.003), 2048: (0.043, 0.040, 0.149, 0.106, 0.004, 0.003),
+    4096: (0.153, 0.098, 0.468, 0.253, 0.007, 0.004), 8192: (0.572, 0.237, 1.699, 0.600, 0.009, 0.004),
+    16384: (2.179, 0.616, 6.455, 1.564, 0.012, 0.005), 32768: (8.570, 1.807, 24.449, 4.358, 0.018, 0.006),
+    65536: (36.431, 5.573, 99.664, 14.150, 0.027, 0.009), 131072: (159.987, 21.758, 441.230, 51.509, 0.045, 0.015),
+}
+
+
+def run_tp_replica(args):
+    """Each rank of a TP=8 group owns one KV head and its 8 QO heads and runs the operator on its
+    shard without any exchange; the group's latency is the slowest rank's.  With fewer than 8 GPUs
+    the shards are timed one after another on the GPUs at hand (rank r takes shards r, r+world, ...):
+    every launch is exactly what that rank's GPU would run.  L2 is flushed before every timed call."""
+    import torch
+    import cowa_inputs
+    import paper_2609_32704_b200 as cowa
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    rank, world, _ = dist_setup(args.gpus)
+    dev = torch.device("cuda", torch.cuda.current_device())
+    TP, Hq_r, D, sink, near = 8, 8, 128, 128, 896
+    scale = cowa_inputs.softmax_scale(D)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    iters = max(args.steps, 3)
+
+    def timed(fn):
+        for _ in range(max(args.warmup, 3)):
+            fn()
+        tot = 0.0
+        for _ in range(iters):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record()
+            torch.cuda.synchronize()
+            tot += e0.elapsed_time(e1)
+        return tot / iters
+
+    rows = []
+    for T in sorted(PAPER_TP8_MS):
+        q, k, v, d_o = cowa_inputs.make_train_inputs(11, 1, T, Hq_r, 1, D, device=dev)
+        o = torch.empty_like(q)
+        lse = torch.empty((1, Hq_r, T), dtype=torch.float32, device=dev)
+        dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+        qd, od = q[:, :, -1].contiguous(), torch.empty((1, Hq_r, D), dtype=torch.bfloat16, device=dev)
+        lsed = torch.empty((1, Hq_r), dtype=torch.float32, device=dev)
+        lens = torch.tensor([T], dtype=torch.int32, device=dev)
+        worst = {}
+        for full in (False, True):
+            for r in range(rank, TP, world):
+                p = cowa.make_params(sink=sink, local=near, softmax_scale=scale, full_attn=full,
+                                     hkv_global=TP, hkv_offset=r)
+                ws = torch.empty(max(cowa.cowa_bwd_workspace_bytes(1, T, Hq_r, 1, D, p), 16), dtype=torch.uint8,
+                                 device=dev)
+                wsd = torch.empty(max(cowa.cowa_decode_workspace_bytes(1, T, Hq_r, 1, D, p), 16), dtype=torch.uint8,
+                                  device=dev)
+                t = {"fwd": timed(lambda: cowa.cowa_fwd(q, k, v, o, lse, p)),
+                     "bwd": timed(lambda: cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, p, ws)),
+                     "dec": timed(lambda: cowa.cowa_decode(qd, k, v, lens, od, lsed, p, wsd))}
+                for ph, ms in t.items():
+                    key = ("full_" if full else "cowa_") + ph
+                    worst[key] = max(worst.get(key, 0.0), ms)
+                if full:
+                    break  # dense shards are identical on every rank
+        cowa.cowa_check_device_status()
+        worst = {k_: max_over_ranks(v_, world) for k_, v_ in sorted(worst.items())}
+        pf, pc, pfb, pcb, pfd, pcd = PAPER_TP8_MS[T]
+        rows.append({"T": T, **{k_ + "_ms": v_ for k_, v_ in worst.items()},
+                     "speedup_fwd": worst["full_fwd"] / worst["cowa_fwd"],
+                     "speedup_bwd": worst["full_bwd"] / worst["cowa_bwd"],
+                     "speedup_dec": worst["full_dec"] / worst["cowa_dec"],
+                     "paper_h100_ms": {"full_fwd": pf, "cowa_fwd": pc, "full_bwd": pfb, "cowa_bwd": pcb,
+                                       "full_dec": pfd, "cowa_dec": pcd}})
+        del q, k, v, d_o, o, lse, dq, dk, dv
+    if rank != 0:
+        return
+    last = rows[-1]
+    print(json.dumps({
+        "metric": "cowa_tp8_shard_fwd_bwd_ms_128k", "value": last["cowa_fwd_ms"] + last["cowa_bwd_ms"], "unit": "ms",
+        "n_gpus": world, "steps": iters, "warmup": max(args.warmup, 3), "higher_is_better": False,
+        "scaling": "strong", "vs_baseline": (last["cowa_fwd_ms"] + last["cowa_bwd_ms"]) / (21.758 + 51.509),
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "TP=8 shards of B=1, Hq=64, Hkv=8, D=128, sink+near=128+896, T=1K..128K",
+                   "shards_per_gpu": TP // world if world <= TP else 1, "l2": "flushed before every timed call",
+                   "latency": "slowest shard (max over the 8 ranks' launches)"},
+        "rows": rows}))
+
+
 BWD_LAUNCHES = 3  # preprocess, main kernel, dq conversion
 
 
@@ -521,6 +615,8 @@ def main():
     ap.add_argument("--no-fullattn", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-varlen", action="store_true")
+    ap.add_argument("--tp-replica", action="store_true",
+                    help="time the TP=8 shards of the paper's operator benchmark shape instead of the default step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--train-cfg", default=TRAIN_CFG, choices=["8k", "32k", "128k"],
@@ -531,6 +627,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.tp_replica:
+        run_tp_replica(args)
     else:
         run_cuda(args)
     if int(os.environ.get("WORLD_SIZE", "1")) > 1:

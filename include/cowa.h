@@ -107,10 +107,13 @@ int cowa_prefill_varlen(const void* q, const void* k, const void* v, void* o, fl
 /* Training backward, Algorithm 2: exact gradient of cowa_fwd.
  *   in: q,k,v,o,lse as produced by cowa_fwd, d_o [B,Hq,T,D];
  *   out: dq [B,Hq,T,D], dk,dv [B,Hkv,T,D] bf16 (fully overwritten).
- * dk,dv are summed over the QO heads of each group inside one thread block (no atomics) and are always
+ * dk,dv are summed over the QO heads of each group inside one thread block, or, when there are too few
+ * (batch, KV head, KV tile) triples to fill the GPU or the sink tiles would dominate, by a few blocks whose
+ * fp32 partial sums a last kernel adds in a fixed order: no atomics (Algorithm 2 line 17 has them), always
  * bitwise reproducible; for dq see cowa_params_t.deterministic.
- * `workspace` (device, >= cowa_bwd_workspace_bytes, 16-byte aligned) holds the fp32
- * row vector rowsum(o*d_o) (Algorithm 2 line 13) and needs no initialisation. */
+ * `workspace` (device, >= cowa_bwd_workspace_bytes for the same B, T, Hq, Hkv, D and params, 16-byte
+ * aligned) holds the fp32 dq accumulator, the row vector rowsum(o*d_o) (Algorithm 2 line 13) and those
+ * partial sums; it needs no initialisation. */
 int cowa_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse,
              const void* d_o, void* dq, void* dk, void* dv,
              int B, int T, int Hq, int Hkv, int D, const cowa_params_t* p,

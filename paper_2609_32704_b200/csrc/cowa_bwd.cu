@@ -49,6 +49,8 @@ struct BwdArgs {
   int B, Nq, Nk, Hq, Hkv, G, Tpad;
   int sink_tiles;      // KV tiles per head that hold sink columns (launched first)
   int dq_fixed;        // 1: dQ partial sums travel as 32-bit fixed point (order-independent addition)
+  int parts;           // blocks per KV tile: each takes G / parts heads of the group (1: the whole group)
+  float* dkv_part;     // parts > 1: fp32 partial dK, dV [B*Hkv, nKV, parts, 2, BKV, D], summed by a last kernel
   float scale, scale_log2;
   CowaHeadWindows wins;
 };
@@ -127,8 +129,9 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 
   // ---- work item: sink tiles of every head first, then head-major with ascending KV tile ----
   int hk, b, j;
+  const int part = blockIdx.x % a.parts;
   {
-    int idx = blockIdx.x;
+    int idx = blockIdx.x / a.parts;
     const int nKV = (a.Nk + BKV - 1) / BKV, nsk = a.sink_tiles, nhead = a.B * a.Hkv;
     if (idx < nsk * nhead) {
       j = idx / nhead; idx %= nhead;
@@ -144,8 +147,10 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   CowaRange rg[2];
   cowa_bwd_ranges(w, k0, k1, off, a.Nq, BQS, rg);
   const int cnt = cowa_range_len(rg[0]) + cowa_range_len(rg[1]);  // QO steps per head
-  const int N = cnt * a.G;
+  const int gs = a.G / a.parts;          // heads of the group handled by this block
+  const int N = cnt * gs;
   const int bhk = b * a.Hkv + hk;
+  const int bhq0 = b * a.Hq + hk * a.G + part * gs;  // first of them
 
   if (tid == 0) {
     mbar_init(bar_kv, 1);
@@ -179,6 +184,30 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     tc_fence_after();
     uint8_t* sOut = sStage + (is_dk ? 0 : SM::kKV);
     const float mul = is_dk ? a.scale : 1.f;
+    if (a.parts > 1) {
+      // The group's heads are spread over several blocks: this block's share goes out in fp32, one slot
+      // per block, and a last kernel adds the slots in a fixed order.
+      const int nKV = (a.Nk + BKV - 1) / BKV;
+      float* dst = a.dkv_part + ((((size_t)bhk * nKV + j) * a.parts + part) * 2 + (is_dk ? 0 : 1)) * (size_t)(BKV * D) +
+                   (size_t)r * D;
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t ov[32];
+        if (N > 0 && ok) {
+          tmem_ld32(t_lane + (is_dk ? cDK : cDV) + c * 32, ov);
+          tmem_wait_ld();
+        } else {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) ov[e] = 0u;
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+          *reinterpret_cast<float4*>(dst + c * 32 + q * 4) =
+              make_float4(__uint_as_float(ov[q * 4]) * mul, __uint_as_float(ov[q * 4 + 1]) * mul,
+                          __uint_as_float(ov[q * 4 + 2]) * mul, __uint_as_float(ov[q * 4 + 3]) * mul);
+      }
+      return;
+    }
 #pragma unroll
     for (int c = 0; c < D / 32; ++c) {
       uint32_t ov[32];
@@ -229,7 +258,7 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           if (n >= NST) ok = mbar_wait(bar_ld_empty + st, ph_e, a.status);
           if (!ok) break;
           const int i = cowa_bwd_tile_at(rg, t_in);
-          const int bhq = b * a.Hq + hk * a.G + g, q0 = i * BQS;
+          const int bhq = bhq0 + g, q0 = i * BQS;
           uint8_t* sQ = sStage + st * SM::kStage;
           uint8_t* sdO = sQ + SM::kQS;
           mbar_expect_tx(bar_ld_full + st, SM::kStage + 512);
@@ -461,7 +490,7 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       int g = 0, t_in = 0;
       for (int n = 0; n < N && ok; ++n) {
         const int i = cowa_bwd_tile_at(rg, t_in);
-        const int bhq = b * a.Hq + hk * a.G + g, q0 = i * BQS;
+        const int bhq = bhq0 + g, q0 = i * BQS;
         if (++t_in == cnt) { t_in = 0; ++g; }
         ok = mbar_wait(bar_dq_full + (n & 1), (n >> 1) & 1, a.status);
         if (!ok) break;
@@ -563,23 +592,94 @@ __global__ void cowa_bwd_convert_dq_kernel(const float* __restrict__ acc, __nv_b
   *reinterpret_cast<uint4*>(dq + ((size_t)bh * T + t) * D + part * 8) = v;
 }
 
+// Sum of the per-block partial dK, dV (heads of a group spread over `parts` blocks), in slot order, to bf16.
+template <int D>
+__global__ void cowa_bwd_reduce_dkv_kernel(const float* __restrict__ part, __nv_bfloat16* __restrict__ dk,
+                                           __nv_bfloat16* __restrict__ dv, int T, int nKV, int parts, long long BHk) {
+  const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;  // one thread per 8 elements of dK and dV
+  const long long total = BHk * nKV * BKV * (D / 8);
+  if (gid >= total) return;
+  const int ch = (int)(gid % (D / 8));
+  const int r = (int)((gid / (D / 8)) % BKV);
+  const long long tile = gid / ((D / 8) * BKV);  // bhk * nKV + j
+  const int j = (int)(tile % nKV);
+  const long long bhk = tile / nKV;
+  const int t = j * BKV + r;
+  if (t >= T) return;
+  float acc[2][8];
+#pragma unroll
+  for (int m = 0; m < 2; ++m)
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[m][e] = 0.f;
+  for (int pi = 0; pi < parts; ++pi)
+#pragma unroll
+    for (int m = 0; m < 2; ++m) {
+      const float4* src = reinterpret_cast<const float4*>(part + (((size_t)tile * parts + pi) * 2 + m) * (size_t)(BKV * D) +
+                                                          (size_t)r * D + ch * 8);
+      const float4 x = src[0], y = src[1];
+      acc[m][0] += x.x; acc[m][1] += x.y; acc[m][2] += x.z; acc[m][3] += x.w;
+      acc[m][4] += y.x; acc[m][5] += y.y; acc[m][6] += y.z; acc[m][7] += y.w;
+    }
+#pragma unroll
+  for (int m = 0; m < 2; ++m) {
+    uint4 v;
+    v.x = pack_bf16(acc[m][0], acc[m][1]); v.y = pack_bf16(acc[m][2], acc[m][3]);
+    v.z = pack_bf16(acc[m][4], acc[m][5]); v.w = pack_bf16(acc[m][6], acc[m][7]);
+    *reinterpret_cast<uint4*>((m == 0 ? dk : dv) + ((size_t)bhk * T + t) * D + ch * 8) = v;
+  }
+}
+
 // Optional CUDA events recorded around the main kernel of the next cowa_bwd calls on this host thread.
 thread_local cudaEvent_t g_ev_main_start = nullptr, g_ev_main_stop = nullptr;
 
-size_t ws_bytes(int B, int T, int Hq, int D) {
+// Blocks per KV tile.  A block normally takes the whole GQA group of its KV tile (dK, dV then never leave
+// TMEM).  That starves the GPU when B * Hkv * tiles is small, and it makes the sink tiles -- visited by
+// every query tile of every head -- the critical path when Hkv is small; in both cases the group's heads
+// are spread over `parts` blocks (a divisor of G), chosen as the smallest that gives two waves of
+// blocks and keeps the longest block under 3/4 of an even share of the work.
+constexpr int kSMs = 148;
+int bwd_parts(int B, int T, int Hkv, int G, const CowaHeadWindows& hw) {
+  const int nKV = (T + BKV - 1) / BKV;
+  long long total = 0, longest = 0;
+  for (int h = 0; h < Hkv; ++h)
+    for (int j = 0; j < nKV; ++j) {
+      CowaRange rg[2];
+      const int k0 = j * BKV, k1 = std::min(k0 + BKV, T) - 1;
+      cowa_bwd_ranges(hw.w[h], k0, k1, 0, T, BQS, rg);
+      const long long cnt = cowa_range_len(rg[0]) + cowa_range_len(rg[1]);
+      total += cnt;
+      longest = std::max(longest, cnt);
+    }
+  total *= (long long)B * G;
+  longest *= G;
+  const long long blocks = (long long)B * Hkv * nKV;
+  for (int p = 1; p < G; ++p) {
+    if (G % p) continue;
+    if (blocks * p >= 2 * kSMs && longest * 4 * kSMs <= 3 * total * p) return p;
+  }
+  return G;
+}
+
+size_t part_bytes(int B, int T, int Hkv, int D, int parts) {
+  if (parts <= 1) return 0;
+  return (size_t)B * Hkv * ((T + BKV - 1) / BKV) * parts * 2 * BKV * D * sizeof(float);
+}
+
+size_t ws_bytes(int B, int T, int Hq, int Hkv, int D, int parts) {
   const size_t Tpad = ((size_t)T + BQS - 1) / BQS * BQS;
-  return (size_t)B * Hq * Tpad * ((size_t)D + 2) * sizeof(float);
+  return (size_t)B * Hq * Tpad * ((size_t)D + 2) * sizeof(float) + part_bytes(B, T, Hkv, D, parts);
 }
 
 template <int D>
 int launch_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* d_o,
                void* dq, void* dk, void* dv, int B, int T, int Hq, int Hkv, const cowa_params_t* p,
-               const CowaHeadWindows& hw, void* ws, cudaStream_t st) {
+               const CowaHeadWindows& hw, int parts, void* ws, cudaStream_t st) {
   const int Tpad = (T + BQS - 1) / BQS * BQS;
   const long long BH = (long long)B * Hq;
   float* dq_acc = static_cast<float*>(ws);
   float* lse2 = dq_acc + (size_t)BH * Tpad * D;
   float* delta = lse2 + (size_t)BH * Tpad;
+  float* dkv_part = delta + (size_t)BH * Tpad;
   COWA_CUDA_TRY(cudaMemsetAsync(dq_acc, 0, (size_t)BH * Tpad * D * sizeof(float), st));
   {
     const long long threads = BH * Tpad * (D / 8);
@@ -608,13 +708,14 @@ int launch_bwd(const void* q, const void* k, const void* v, const void* o, const
   a.wins = hw;
   a.sink_tiles = 0;
   a.dq_fixed = p->deterministic ? 1 : 0;
+  a.parts = parts; a.dkv_part = dkv_part;
   for (int h = 0; h < Hkv; ++h) {
     const int sk = hw.w[h].s < T ? hw.w[h].s : T;
     a.sink_tiles = std::max(a.sink_tiles, (sk + BKV - 1) / BKV);
   }
   COWA_CUDA_TRY(cudaFuncSetAttribute(cowa_bwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      BwdSmem<D>::kBytes));
-  const long long nblocks = (long long)((T + BKV - 1) / BKV) * B * Hkv;
+  const long long nblocks = (long long)((T + BKV - 1) / BKV) * B * Hkv * parts;
   if (nblocks > 0x7FFFFFFFll) return COWA_ERR_UNSUPPORTED;
   if (g_ev_main_start) COWA_CUDA_TRY(cudaEventRecord(g_ev_main_start, st));
   cowa_bwd_kernel<D><<<(unsigned)nblocks, 512, BwdSmem<D>::kBytes, st>>>(mq, mk, mv, mdo, mdk, mdv, mdq, a);
@@ -624,6 +725,13 @@ int launch_bwd(const void* q, const void* k, const void* v, const void* o, const
     const long long threads = BH * T * (D / 8);
     cowa_bwd_convert_dq_kernel<D><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(
         dq_acc, static_cast<__nv_bfloat16*>(dq), T, Tpad, BH, p->deterministic ? 1 : 0);
+    COWA_CUDA_TRY(cudaGetLastError());
+  }
+  if (parts > 1) {
+    const int nKV = (T + BKV - 1) / BKV;
+    const long long threads = (long long)B * Hkv * nKV * BKV * (D / 8);
+    cowa_bwd_reduce_dkv_kernel<D><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(
+        dkv_part, static_cast<__nv_bfloat16*>(dk), static_cast<__nv_bfloat16*>(dv), T, nKV, parts, (long long)B * Hkv);
     COWA_CUDA_TRY(cudaGetLastError());
   }
   return COWA_OK;
@@ -640,9 +748,10 @@ int cowa_bwd_set_profile_events(void* start_event, void* stop_event) {
 }
 
 size_t cowa_bwd_workspace_bytes(int B, int T, int Hq, int Hkv, int D, const cowa_params_t* p) {
-  (void)Hkv; (void)p;
-  if (B <= 0 || T <= 0 || Hq <= 0 || D <= 0) return 0;
-  return ws_bytes(B, T, Hq, D);
+  if (B <= 0 || T <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || D <= 0 || !p) return 0;
+  CowaHeadWindows hw;
+  if (cowa::resolve_windows(T, Hkv, p, &hw) != COWA_OK) return 0;
+  return ws_bytes(B, T, Hq, Hkv, D, bwd_parts(B, T, Hkv, Hq / Hkv, hw));
 }
 
 int cowa_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* d_o,
@@ -655,13 +764,14 @@ int cowa_bwd(const void* q, const void* k, const void* v, const void* o, const f
   const void* ptrs[] = {q, k, v, o, d_o, dq, dk, dv, workspace};
   for (const void* x : ptrs)
     if (!cowa::aligned16(x)) return COWA_ERR_MISALIGNED;
-  if (workspace_bytes < ws_bytes(B, T, Hq, D)) return COWA_ERR_WORKSPACE_TOO_SMALL;
   CowaHeadWindows hw;
   int rc = cowa::resolve_windows(T, Hkv, p, &hw);
   if (rc != COWA_OK) return rc;
+  const int parts = bwd_parts(B, T, Hkv, Hq / Hkv, hw);
+  if (workspace_bytes < ws_bytes(B, T, Hq, Hkv, D, parts)) return COWA_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  return D == 128 ? launch_bwd<128>(q, k, v, o, lse, d_o, dq, dk, dv, B, T, Hq, Hkv, p, hw, workspace, st)
-                  : launch_bwd<64>(q, k, v, o, lse, d_o, dq, dk, dv, B, T, Hq, Hkv, p, hw, workspace, st);
+  return D == 128 ? launch_bwd<128>(q, k, v, o, lse, d_o, dq, dk, dv, B, T, Hq, Hkv, p, hw, parts, workspace, st)
+                  : launch_bwd<64>(q, k, v, o, lse, d_o, dq, dk, dv, B, T, Hq, Hkv, p, hw, parts, workspace, st);
 }
 
 }  // extern "C"

@@ -295,6 +295,46 @@ def test_bwd_full_attn_and_explicit_windows():
     bwd_case(1, 700, 2, 2, 128, 0, 1, windows=[(0, 50, 100, 200), (20, 10, 0, 0)])
 
 
+def _bwd_blocks_per_tile(B, T, Hq, Hkv, D, params):
+    """How many blocks share a KV tile's GQA group, read off the workspace size."""
+    tpad = (T + 63) // 64 * 64
+    extra = cowa.cowa_bwd_workspace_bytes(B, T, Hq, Hkv, D, params) - B * Hq * tpad * (D + 2) * 4
+    per = B * Hkv * ((T + 127) // 128) * 2 * 128 * D * 4
+    assert extra % per == 0
+    return max(extra // per, 1)
+
+
+def test_bwd_tensor_parallel_shard():
+    # One KV head of eight and its 8 QO heads, as a TP=8 rank holds them: windows of the global head, and
+    # (few blocks, long sink tiles) the group's heads spread over several blocks per KV tile.
+    T, Hq, D, sink, local = 3000, 8, 128, 40, 200
+    scale = cowa_inputs.softmax_scale(D)
+    for r in (0, 5):
+        q, k, v, d_o = cowa_inputs.make_train_inputs(56 + r, 1, T, Hq, 1, D)
+        params = cowa.make_params(sink=sink, local=local, softmax_scale=scale, hkv_global=8, hkv_offset=r)
+        assert _bwd_blocks_per_tile(1, T, Hq, 1, D, params) == 8
+        dq, dk, dv = run_fwd_bwd(q.to(DEV), k.to(DEV), v.to(DEV), d_o.to(DEV), params)
+        ws = orc.default_windows(T, 8, sink, local)[r:r + 1]
+        f = cowa_inputs.to_f64
+        dq_r, dk_r, dv_r = orc.backward(f(q[0]), f(k[0]), f(v[0]), f(d_o[0]), ws, scale)
+        check_grad(f"shard {r} dq", dq[0].float().cpu().numpy(), dq_r)
+        check_grad(f"shard {r} dk", dk[0].float().cpu().numpy(), dk_r)
+        check_grad(f"shard {r} dv", dv[0].float().cpu().numpy(), dv_r)
+
+
+def test_bwd_group_split_over_some_blocks():
+    # A shape where the group of 8 heads is split over 4 blocks of 2 heads each; dK, dV stay bitwise
+    # repeatable because the partial sums are added in slot order.
+    B, T, Hq, Hkv, D, sink, local = 4, 2048, 16, 2, 64, 16, 256
+    params = cowa.make_params(sink=sink, local=local, softmax_scale=cowa_inputs.softmax_scale(D))
+    assert _bwd_blocks_per_tile(B, T, Hq, Hkv, D, params) == 4
+    bwd_case(B, T, Hq, Hkv, D, sink, local, seed=58)
+    q, k, v, d_o = cowa_inputs.make_train_inputs(58, B, T, Hq, Hkv, D, device=DEV)
+    _, dk1, dv1 = run_fwd_bwd(q, k, v, d_o, params)
+    _, dk2, dv2 = run_fwd_bwd(q, k, v, d_o, params)
+    assert torch.equal(dk1, dk2) and torch.equal(dv1, dv2)
+
+
 def test_bwd_dkdv_bitwise_repeatable():
     # dK and dV are accumulated in a fixed order inside one block: two runs must agree bit for bit.
     q, k, v, d_o = cowa_inputs.make_train_inputs(52, 1, 2048, 8, 2, 128, device=DEV)
