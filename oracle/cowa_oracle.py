@@ -60,6 +60,38 @@ def default_windows(n_k, h_k_global, w_sink, w_near, hk_offset=0, hk_local=None)
     ]
 
 
+def equal_area_windows(n_q, n_k, h_k_global, w_sink, w_near, hk_offset=0, hk_local=None):
+    """Equal-area breakpoints: another breakpoint schedule under the same support rule
+    (Eq. fwa_support; Sec. 2.1 notes that other schedules redistribute long-range work and
+    leaves equal-area allocation for training out of its scope, so the rule is this build's).
+
+    The band offset x (distance delta = w_near + x, 0 <= x < L) is weighted by the number of
+    queries for which that distance is causal and points at a key outside the sink:
+        c(x) = #{ i_q in [0, N_q) : i_q + (N_k - N_q) - (w_near + x) >= w_sink },
+    W(b) = sum_{x < b} c(x), and b_h is the smallest b with H_k * W(b) >= h * W(L), h = 0..H_k.
+    The tuples have the default pattern's form (w_sink, w_near, b_h, b_{h+1} - b_h)."""
+    if hk_local is None:
+        hk_local = h_k_global - hk_offset
+    n_q, n_k, w_sink, w_near = int(n_q), int(n_k), int(w_sink), int(w_near)
+    span = max(n_k - w_sink - w_near, 0)
+    off = n_k - n_q
+    x = np.arange(span, dtype=np.int64)
+    first_query = np.maximum(w_near + x + w_sink - off, 0)  # first query that reaches a non-sink key
+    c = np.clip(n_q - first_query, 0, n_q)
+    cum = np.concatenate([[0], np.cumsum(c)]).astype(object)  # exact integers
+    total = cum[-1]
+    b = []
+    for h in range(h_k_global + 1):
+        lo = 0
+        while h_k_global * cum[lo] < h * total:  # plain scan: obviously the smallest such b
+            lo += 1
+        b.append(lo)
+    return [
+        (w_sink, w_near, b[g], b[g + 1] - b[g])
+        for g in range(hk_offset, hk_offset + hk_local)
+    ]
+
+
 def duplicated_windows(n_k, h_k, w_sink, w_near, m):
     """m-unique-window control layout (App. A.1): the m long-range regions
     nearest the near window, W_1..W_m of the H_k-way split, are repeated over

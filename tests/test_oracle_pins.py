@@ -132,6 +132,61 @@ def test_breakpoints_floor_and_global_index():
 
 # ---------------------------------------------------------------- forward
 
+# ---------------------------------------------------------------- equal-area breakpoints
+
+@pytest.mark.parametrize("n_q,n_k,h_k,sink,near", [
+    (90, 90, 4, 3, 10), (64, 150, 3, 5, 7), (200, 200, 8, 0, 1), (1, 77, 5, 2, 6), (120, 120, 2, 100, 30),
+])
+def test_equal_area_windows_balance_and_coverage(n_q, n_k, h_k, sink, near):
+    ws = orc.equal_area_windows(n_q, n_k, h_k, sink, near)
+    span = max(n_k - sink - near, 0)
+    # same shape as the default pattern: shared sink/near, bands tile [0, L) in order without gaps
+    assert [w[:2] for w in ws] == [(sink, near)] * h_k
+    assert ws[0][2] == 0 and all(ws[h][2] + ws[h][3] == ws[h + 1][2] for h in range(h_k - 1))
+    assert ws[-1][2] + ws[-1][3] == span
+    # hence the heads still cover the whole causal prefix together (Eq. fwa_collective_coverage)
+    union = np.zeros((n_q, n_k), dtype=bool)
+    for w in ws:
+        union |= orc.visible_mask(n_q, n_k, w)
+    iq, ik = np.meshgrid(np.arange(n_q), np.arange(n_k), indexing="ij")
+    assert np.array_equal(union, iq + (n_k - n_q) - ik >= 0)
+    if span == 0:
+        return
+    # brute force on the explicit masks: the pairs a band adds outside sink and near window, per head
+    # and cumulatively; every breakpoint is the first offset whose cumulative count reaches h/H of the total
+    delta = iq + (n_k - n_q) - ik
+    outside = (delta >= near) & (ik >= sink)
+    per_offset = np.array([int((outside & (delta == near + x)).sum()) for x in range(span)])
+    cum = np.concatenate([[0], np.cumsum(per_offset)])
+    for h, w in enumerate(ws):
+        b = w[2]
+        assert h_k * cum[b] >= h * cum[-1]
+        assert b == 0 or h_k * cum[b - 1] < h * cum[-1]
+    areas = [int(cum[w[2] + w[3]] - cum[w[2]]) for w in ws]
+    assert sum(areas) == cum[-1]
+    assert max(areas) - min(areas) <= 2 * per_offset.max()  # balanced to within the heaviest diagonals
+
+
+def test_equal_area_windows_special_cases():
+    # one query (decode): every offset weighs 1, so equal area is equal width, b_h = ceil(h L / H)
+    n_k, h_k, sink, near = 1000, 7, 11, 40
+    span = n_k - sink - near
+    ws = orc.equal_area_windows(1, n_k, h_k, sink, near)
+    assert [w[2] for w in ws] == [-(-h * span // h_k) for h in range(h_k)]
+    # square causal case: offsets weigh L, L-1, ..., 1 (a triangle); cutting a triangle into H equal
+    # areas from its long side puts the cuts at L (1 - sqrt(1 - h/H))
+    n, h_k = 40000, 8
+    ws = orc.equal_area_windows(n, n, h_k, 0, 1)
+    span = n - 1
+    for h, w in enumerate(ws):
+        assert abs(w[2] - span * (1.0 - np.sqrt(1.0 - h / h_k))) <= 1.0
+    # global head indexing: a rank's tuples are a slice of the global list
+    full = orc.equal_area_windows(500, 800, 6, 9, 20)
+    assert orc.equal_area_windows(500, 800, 6, 9, 20, hk_offset=2, hk_local=3) == full[2:5]
+    # sink + near already cover everything: no bands
+    assert orc.equal_area_windows(50, 50, 4, 30, 30) == [(30, 30, 0, 0)] * 4
+
+
 def _rand(h_q, h_k, n_q, n_k, d):
     q = RNG.standard_normal((h_q, n_q, d))
     k = RNG.standard_normal((h_k, n_k, d))
