@@ -563,21 +563,26 @@ def run_tp_replica(args):
         lsed = torch.empty((1, Hq_r), dtype=torch.float32, device=dev)
         lens = torch.tensor([T], dtype=torch.int32, device=dev)
         worst = {}
-        for full in (False, True):
+        for layout in ("cowa", "eq", "full"):  # default equal-width bands, equal-area bands, dense
             for r in range(rank, TP, world):
-                p = cowa.make_params(sink=sink, local=near, softmax_scale=scale, full_attn=full,
-                                     hkv_global=TP, hkv_offset=r)
+                if layout == "eq":
+                    p = cowa.make_params(windows=cowa.cowa_equal_area_windows(T, T, TP, r, 1, sink, near),
+                                         softmax_scale=scale)
+                else:
+                    p = cowa.make_params(sink=sink, local=near, softmax_scale=scale, full_attn=(layout == "full"),
+                                         hkv_global=TP, hkv_offset=r)
                 ws = torch.empty(max(cowa.cowa_bwd_workspace_bytes(1, T, Hq_r, 1, D, p), 16), dtype=torch.uint8,
                                  device=dev)
                 wsd = torch.empty(max(cowa.cowa_decode_workspace_bytes(1, T, Hq_r, 1, D, p), 16), dtype=torch.uint8,
                                   device=dev)
                 t = {"fwd": timed(lambda: cowa.cowa_fwd(q, k, v, o, lse, p)),
-                     "bwd": timed(lambda: cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, p, ws)),
-                     "dec": timed(lambda: cowa.cowa_decode(qd, k, v, lens, od, lsed, p, wsd))}
+                     "bwd": timed(lambda: cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, p, ws))}
+                if layout != "eq":  # decode keeps the equal-width rule (Sec. 2.1), so there is no third variant
+                    t["dec"] = timed(lambda: cowa.cowa_decode(qd, k, v, lens, od, lsed, p, wsd))
                 for ph, ms in t.items():
-                    key = ("full_" if full else "cowa_") + ph
+                    key = layout + "_" + ph
                     worst[key] = max(worst.get(key, 0.0), ms)
-                if full:
+                if layout == "full":
                     break  # dense shards are identical on every rank
         cowa.cowa_check_device_status()
         worst = {k_: max_over_ranks(v_, world) for k_, v_ in sorted(worst.items())}
@@ -585,6 +590,8 @@ def run_tp_replica(args):
         rows.append({"T": T, **{k_ + "_ms": v_ for k_, v_ in worst.items()},
                      "speedup_fwd": worst["full_fwd"] / worst["cowa_fwd"],
                      "speedup_bwd": worst["full_bwd"] / worst["cowa_bwd"],
+                     "speedup_fwd_equal_area": worst["full_fwd"] / worst["eq_fwd"],
+                     "speedup_bwd_equal_area": worst["full_bwd"] / worst["eq_bwd"],
                      "speedup_dec": worst["full_dec"] / worst["cowa_dec"],
                      "paper_h100_ms": {"full_fwd": pf, "cowa_fwd": pc, "full_bwd": pfb, "cowa_bwd": pcb,
                                        "full_dec": pfd, "cowa_dec": pcd}})

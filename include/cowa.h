@@ -174,6 +174,18 @@ size_t cowa_decode_workspace_bytes(int B, int Tmax, int Hq, int Hkv, int D, cons
 int cowa_default_windows(int Nk, int Hkv_global, int hkv_offset, int Hkv_local,
                          int sink, int local, cowa_window_t* out);
 
+/* Host-only.  Equal-area breakpoints for training / prefill: tuples of the same form
+ * (sink, local, b_h, b_{h+1}-b_h) whose bands still tile [0, L), so collective coverage
+ * (Eq. fwa_collective_coverage) holds, but with the breakpoints moved so that every head's band holds
+ * about the same number of legal (query, key) pairs.  Sec. 2.1 allows other breakpoint schedules under
+ * the same support rule and leaves equal-area allocation out of its scope: the rule below is this
+ * library's.  Band offset x (distance local + x) weighs c(x) = number of queries i_q in [0, Nq) with
+ * i_q + (Nk - Nq) - (local + x) >= sink; W(b) = sum_{x<b} c(x); b_h = the smallest b with
+ * Hkv_global * W(b) >= h * W(L).  Pass the result as cowa_params_t.windows.  out: HOST array of Hkv_local
+ * tuples for global heads hkv_offset .. hkv_offset+Hkv_local-1.  Cost O(L). */
+int cowa_equal_area_windows(int Nq, int Nk, int Hkv_global, int hkv_offset, int Hkv_local,
+                            int sink, int local, cowa_window_t* out);
+
 /* Host-only.  Writes the analytic tile schedule (Sec. 2.3: block sets J_h(i), I_h(j)) that the
  * kernels' scheduler computes, as an int32 stream into the HOST buffer `out`:
  *   COWA_SCHED_FWD    for each head h, QO tile i:  h, i, n, then n pairs (j, full) with j descending

@@ -68,6 +68,8 @@ def lib():
         L.cowa_decode_workspace_bytes.restype = sz
         L.cowa_default_windows.argtypes = [i32] * 6 + [C.POINTER(Window)]
         L.cowa_default_windows.restype = i32
+        L.cowa_equal_area_windows.argtypes = [i32] * 7 + [C.POINTER(Window)]
+        L.cowa_equal_area_windows.restype = i32
         L.cowa_schedule_dump.argtypes = [i32, i32, i32, i32, pp, C.POINTER(C.c_int32), sz, C.POINTER(sz)]
         L.cowa_schedule_dump.restype = i32
         L.cowa_tile_counts.argtypes = [i32, i32, i32, pp, C.POINTER(C.c_int64)]
@@ -230,6 +232,13 @@ def cowa_default_windows(Nk, Hkv_global, hkv_offset, Hkv_local, sink, local):
     out = (Window * Hkv_local)()
     _check(lib().cowa_default_windows(Nk, Hkv_global, hkv_offset, Hkv_local, sink, local, out),
            "cowa_default_windows")
+    return [(w.sink, w.near, w.gap, w.len) for w in out]
+
+
+def cowa_equal_area_windows(Nq, Nk, Hkv_global, hkv_offset, Hkv_local, sink, local):
+    out = (Window * Hkv_local)()
+    _check(lib().cowa_equal_area_windows(Nq, Nk, Hkv_global, hkv_offset, Hkv_local, sink, local, out),
+           "cowa_equal_area_windows")
     return [(w.sink, w.near, w.gap, w.len) for w in out]
 
 

@@ -2,6 +2,8 @@
 // tile counts, status reporting.
 #include <string.h>
 
+#include <algorithm>
+#include <vector>
 #include "cowa_common.h"
 
 namespace {
@@ -64,6 +66,36 @@ int cowa_default_windows(int Nk, int Hkv_global, int hkv_offset, int Hkv_local, 
   for (int h = 0; h < Hkv_local; ++h) {
     CowaWin w = cowa_default_window(Nk, Hkv_global, hkv_offset + h, sink, local);
     out[h].sink = w.s; out[h].near = w.n; out[h].gap = w.g; out[h].len = w.l;
+  }
+  return COWA_OK;
+}
+
+int cowa_equal_area_windows(int Nq, int Nk, int Hkv_global, int hkv_offset, int Hkv_local, int sink, int local,
+                            cowa_window_t* out) {
+  if (!out || Nq <= 0 || Nk < Nq || Hkv_global <= 0 || Hkv_local <= 0 || hkv_offset < 0 ||
+      hkv_offset + Hkv_local > Hkv_global || sink < 0 || local < 1)
+    return COWA_ERR_INVALID_ARG;
+  const long long L = std::max((long long)Nk - sink - local, 0ll);
+  const long long off = (long long)Nk - Nq;
+  // queries that reach a key outside the sink at band offset x (distance local + x)
+  auto weight = [&](long long x) {
+    const long long first = std::max(local + x + sink - off, 0ll);
+    return std::min(std::max((long long)Nq - first, 0ll), (long long)Nq);
+  };
+  unsigned __int128 total = 0;
+  for (long long x = 0; x < L; ++x) total += (unsigned long long)weight(x);
+  // one sweep: b_h = first b whose cumulative weight, times H, reaches h * total
+  std::vector<long long> b(Hkv_global + 1, L);
+  unsigned __int128 cum = 0;
+  long long x = 0;
+  for (int h = 0; h <= Hkv_global; ++h) {
+    while ((unsigned __int128)Hkv_global * cum < (unsigned __int128)h * total) cum += (unsigned long long)weight(x++);
+    b[h] = x;
+  }
+  for (int h = 0; h < Hkv_local; ++h) {
+    const int g = hkv_offset + h;
+    out[h].sink = sink; out[h].near = local;
+    out[h].gap = (int32_t)b[g]; out[h].len = (int32_t)(b[g + 1] - b[g]);
   }
   return COWA_OK;
 }

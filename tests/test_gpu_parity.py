@@ -335,6 +335,15 @@ def test_bwd_group_split_over_some_blocks():
     assert torch.equal(dk1, dk2) and torch.equal(dv1, dv2)
 
 
+def test_fwd_bwd_equal_area_windows():
+    # the library's equal-area breakpoints passed back as explicit tuples (training shape, ragged tail)
+    T, Hq, Hkv, D, sink, local = 1900, 8, 4, 128, 24, 100
+    ws = cowa.cowa_equal_area_windows(T, T, Hkv, 0, Hkv, sink, local)
+    assert ws == orc.equal_area_windows(T, T, Hkv, sink, local)
+    fwd_case(1, T, Hq, Hkv, D, sink, local, seed=59, windows=ws)
+    bwd_case(1, T, Hq, Hkv, D, sink, local, seed=59, windows=ws)
+
+
 def test_bwd_dkdv_bitwise_repeatable():
     # dK and dV are accumulated in a fixed order inside one block: two runs must agree bit for bit.
     q, k, v, d_o = cowa_inputs.make_train_inputs(52, 1, 2048, 8, 2, 128, device=DEV)

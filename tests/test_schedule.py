@@ -130,6 +130,43 @@ def test_schedule_benchmark_configs_sampled(name):
     assert cnt["causal"] == Hkv * nt * (nt + 1) // 2
 
 
+def test_equal_area_windows_match_oracle():
+    rng = np.random.default_rng(99)
+    cases = [(131072, 131072, 8, 128, 896), (32768, 32768, 8, 128, 2048), (1, 5000, 7, 3, 50),
+             (50, 50, 4, 30, 30), (64, 150, 3, 5, 7)]
+    for _ in range(60):
+        nk = int(rng.integers(1, 5000))
+        nq = int(rng.integers(1, nk + 1))
+        cases.append((nq, nk, int(rng.integers(1, 17)), int(rng.integers(0, 300)), int(rng.integers(1, 600))))
+    for nq, nk, hk, sink, near in cases:
+        want = orc.equal_area_windows(nq, nk, hk, sink, near)
+        assert cowa.cowa_equal_area_windows(nq, nk, hk, 0, hk, sink, near) == want, (nq, nk, hk, sink, near)
+        lo = hk // 3
+        assert cowa.cowa_equal_area_windows(nq, nk, hk, lo, hk - lo, sink, near) == want[lo:]
+    with pytest.raises(cowa.CowaError):
+        cowa.cowa_equal_area_windows(10, 5, 2, 0, 2, 0, 1)      # N_q > N_k
+    with pytest.raises(cowa.CowaError):
+        cowa.cowa_equal_area_windows(10, 10, 2, 1, 2, 0, 1)     # heads beyond the global count
+
+
+def test_equal_area_schedule_balances_visited_tiles():
+    """With the equal-area tuples passed as explicit windows, the visited-tile counts of the heads
+    (128K benchmark shape of one TP group) are within a few percent of each other, while the default
+    equal-width bands differ by a factor of several."""
+    T, hk, sink, near = 131072, 8, 128, 896
+    def per_head(ws):
+        out = []
+        for w in ws:
+            p = cowa.make_params(windows=[w], softmax_scale=1.0)
+            out.append(cowa.cowa_tile_counts(T, T, 1, p)["visited"])
+        return out
+    eq = per_head(cowa.cowa_equal_area_windows(T, T, hk, 0, hk, sink, near))
+    df = per_head(cowa.cowa_default_windows(T, hk, 0, hk, sink, near))
+    assert max(eq) / min(eq) < 1.05
+    assert max(df) / min(df) > 3.0
+    assert abs(sum(eq) - sum(df)) / sum(df) < 0.02   # same total work, redistributed
+
+
 def test_decode_schedule():
     for Nk, Hkv, sink, near, Bk in [(131072, 8, 128, 4096, 128), (98304, 8, 128, 4096, 128),
                                     (100001, 8, 128, 4096, 128), (777, 4, 5, 60, 64), (50, 8, 30, 30, 16),
