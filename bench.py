@@ -319,6 +319,50 @@ def run_cuda(args):
     barrier(world)
     dec_b2b_ms = max_over_ranks(eb[0].elapsed_time(eb[1]) / n_dec, world)
 
+    # ---- decode variants on the same cache: several newest tokens per call, paged cache ----
+    dec_var = None
+    if not args.no_varlen:
+        def b2b(fn):
+            for _ in range(3):
+                fn()
+            ev3 = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+            ev3[0].record()
+            for _ in range(n_dec):
+                fn()
+            ev3[1].record()
+            torch.cuda.synchronize()
+            return max_over_ranks(ev3[0].elapsed_time(ev3[1]) / n_dec, world)
+
+        dec_var = {}
+        Bd, Hqd, Hkvd, Dd, Tm = cd["B"], cd["Hq"], cd["Hkv"], cd["D"], cd["Tmax"]
+        for nq in (2, 4):
+            qm = cowa_inputs.make_train_inputs(9, Bd, nq, Hqd, Hkvd, Dd, device=dev)[0].permute(0, 2, 1, 3).contiguous()
+            om = torch.empty_like(qm)
+            wsm = torch.empty(cowa.cowa_decode_multi_workspace_bytes(Bd, nq, Tm, Hqd, Hkvd, Dd, p_dec),
+                              dtype=torch.uint8, device=dev)
+            ms = b2b(lambda: cowa.cowa_decode_multi(qm, kc, vc, lens, om, None, p_dec, wsm))
+            dec_var[f"multi_nq{nq}"] = {"us_per_call": ms * 1e3, "us_per_token": ms * 1e3 / (Bd * nq),
+                                        "visible_kv_gbs": dec_bytes / (ms * 1e-3) / 1e9}
+        ps = 64
+        mp = Tm // ps
+        perm = torch.randperm(Bd * mp, generator=torch.Generator().manual_seed(5)).to(dev)
+        table = perm.view(Bd, mp).to(torch.int32).contiguous()
+        def to_pages(x):
+            pages = x.view(Bd, Hkvd, mp, ps, Dd).permute(0, 2, 1, 3, 4).reshape(Bd * mp, Hkvd, ps, Dd)
+            out = torch.empty_like(pages)
+            out[perm] = pages
+            return out
+        kp, vp = to_pages(kc), to_pages(vc)
+        q1 = qd.view(Bd, 1, Hqd, Dd)
+        o1 = torch.empty_like(q1)
+        wsp = torch.empty(cowa.cowa_decode_multi_workspace_bytes(Bd, 1, Tm, Hqd, Hkvd, Dd, p_dec), dtype=torch.uint8,
+                          device=dev)
+        ms = b2b(lambda: cowa.cowa_decode_paged(q1, kp, vp, table, lens, o1, None, p_dec, wsp))
+        dec_var[f"paged_{ps}"] = {"us_per_call": ms * 1e3, "visible_kv_gbs": dec_bytes / (ms * 1e-3) / 1e9,
+                                  "max_abs_diff_vs_contiguous": float((o1.view_as(od).float() - od.float()).abs().max())}
+        cowa.cowa_check_device_status()
+        del kp, vp
+
     # ---- FullAttn path of the same library (few iterations: it is ~5.4x the work) ----
     full = {}
     if rank == 0 and not args.no_fullattn:
@@ -502,7 +546,7 @@ def run_cuda(args):
         "bwd_ms": bwd_ms if have_bwd else None, "bwd_tflops": bwd_flops / bwd_ms / 1e9 if have_bwd else None,
         "bwd_main_kernel_ms": bwd_main_ms,
         "visited_tiles": cnt["visited"], "causal_tiles": cnt["causal"],
-        "decode": decode, "prefill_varlen": varlen, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
+        "decode": decode, "prefill_varlen": varlen, "decode_variants": dec_var, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
         "gpu_launches": args.steps * (1 + (BWD_LAUNCHES if have_bwd else 0) + 2),
     }
     line.update(full)

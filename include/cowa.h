@@ -165,6 +165,33 @@ int cowa_decode_static(const void* q, const void* kcache, const void* vcache, co
                        const cowa_params_t* p, void* stream);
 size_t cowa_decode_static_capacity(void);
 
+/* Decode of the Nq newest tokens of every sequence in one call (speculative / multi-token decoding).
+ * The paper's decode step is the forward with N_q = 1 (Sec. 2.3 "Decoding"); this is the same forward with
+ * N_q = Nq: token t of sequence b sits at key position lens[b] - Nq + t, sees keys by Eq. fwa_support at its
+ * own distance (Eq. fwa_distance with N_k = lens[b]), and the windows are built from lens[b] for all Nq
+ * tokens alike.  The paper describes no such variant; the distance rule is unchanged.
+ *   q [B,Nq,Hq,D] in; o [B,Nq,Hq,D] bf16 and lse [B,Nq,Hq] fp32 (may be NULL) out;
+ *   kcache, vcache [B,Hkv,Tmax,D] already hold the Nq new tokens; lens: DEVICE int32[B], Nq <= lens[b] <= Tmax.
+ * 1 <= Nq <= 64; Hq/Hkv in {1,2,4,8}.  Tokens are packed into the 8 columns of the score MMA together with
+ * the group's heads: 8/(Hq/Hkv) tokens share one pass over the visible rows, more tokens take more blocks
+ * (their re-reads mostly hit in L2).  `workspace`: device, >= cowa_decode_multi_workspace_bytes, 16-byte
+ * aligned, no initialisation needed.  cowa_params_t.windows is ignored, as in cowa_decode. */
+int cowa_decode_multi(const void* q, const void* kcache, const void* vcache, const int32_t* lens,
+                      void* o, float* lse, int B, int Nq, int Tmax, int Hq, int Hkv, int D,
+                      const cowa_params_t* p, void* workspace, size_t workspace_bytes, void* stream);
+
+/* The same over a paged KV cache (not in the paper: a serving-side memory layout).
+ *   kpages, vpages [num_pages, Hkv, page_size, D] bf16; block_table: DEVICE int32 [B, max_pages], entry
+ *   [b, i] = page holding tokens [i*page_size, (i+1)*page_size) of sequence b (entries past the sequence's
+ *   last page are not read); page_size a multiple of 16; lens[b] <= max_pages * page_size.
+ * Other arguments, Nq included (Nq = 1 is plain paged decode), as for cowa_decode_multi; workspace size from
+ * cowa_decode_multi_workspace_bytes with Tmax = max_pages * page_size.  Page indices are not range-checked. */
+int cowa_decode_paged(const void* q, const void* kpages, const void* vpages, const int32_t* block_table,
+                      const int32_t* lens, void* o, float* lse, int B, int Nq, int max_pages, int page_size,
+                      int Hq, int Hkv, int D, const cowa_params_t* p, void* workspace, size_t workspace_bytes,
+                      void* stream);
+size_t cowa_decode_multi_workspace_bytes(int B, int Nq, int Tmax, int Hq, int Hkv, int D, const cowa_params_t* p);
+
 size_t cowa_bwd_workspace_bytes(int B, int T, int Hq, int Hkv, int D, const cowa_params_t* p);
 size_t cowa_decode_workspace_bytes(int B, int Tmax, int Hq, int Hkv, int D, const cowa_params_t* p);
 

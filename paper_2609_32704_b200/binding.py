@@ -58,6 +58,12 @@ def lib():
         L.cowa_decode.restype = i32
         L.cowa_decode_static.argtypes = [vp] * 6 + [i32] * 5 + [pp, vp]
         L.cowa_decode_static.restype = i32
+        L.cowa_decode_multi.argtypes = [vp] * 6 + [i32] * 6 + [pp, vp, sz, vp]
+        L.cowa_decode_multi.restype = i32
+        L.cowa_decode_paged.argtypes = [vp] * 7 + [i32] * 7 + [pp, vp, sz, vp]
+        L.cowa_decode_paged.restype = i32
+        L.cowa_decode_multi_workspace_bytes.argtypes = [i32] * 6 + [pp]
+        L.cowa_decode_multi_workspace_bytes.restype = sz
         L.cowa_decode_static_capacity.argtypes = []
         L.cowa_decode_static_capacity.restype = sz
         L.cowa_bwd_set_profile_events.argtypes = [vp, vp]
@@ -210,6 +216,44 @@ def cowa_decode(q, kcache, vcache, lens, o, lse, params, workspace):
 
 def cowa_decode_static_capacity():
     return int(lib().cowa_decode_static_capacity())
+
+
+def cowa_decode_multi_workspace_bytes(B, Nq, Tmax, Hq, Hkv, D, params):
+    return int(lib().cowa_decode_multi_workspace_bytes(B, Nq, Tmax, Hq, Hkv, D, C.byref(params)))
+
+
+def cowa_decode_multi(q, kcache, vcache, lens, o, lse, params, workspace):
+    """q, o [B,Nq,Hq,D]; kcache/vcache [B,Hkv,Tmax,D]; lens int32 [B] (device); lse [B,Nq,Hq] or None."""
+    import torch
+    for t, n in ((q, "q"), (kcache, "kcache"), (vcache, "vcache"), (o, "o")):
+        _need(t, torch.bfloat16, n)
+    _need(lens, torch.int32, "lens")
+    if lse is not None:
+        _need(lse, torch.float32, "lse")
+    B, Nq, Hq, D = q.shape
+    Hkv, Tmax = kcache.shape[1], kcache.shape[2]
+    _check(lib().cowa_decode_multi(_ptr(q), _ptr(kcache), _ptr(vcache), _ptr(lens), _ptr(o),
+                                   _ptr(lse) if lse is not None else None, B, Nq, Tmax, Hq, Hkv, D, C.byref(params),
+                                   _ptr(workspace), workspace.numel() * workspace.element_size(), _stream()),
+           "cowa_decode_multi")
+
+
+def cowa_decode_paged(q, kpages, vpages, block_table, lens, o, lse, params, workspace):
+    """q, o [B,Nq,Hq,D]; kpages/vpages [num_pages,Hkv,page_size,D]; block_table int32 [B,max_pages] (device)."""
+    import torch
+    for t, n in ((q, "q"), (kpages, "kpages"), (vpages, "vpages"), (o, "o")):
+        _need(t, torch.bfloat16, n)
+    _need(lens, torch.int32, "lens")
+    _need(block_table, torch.int32, "block_table")
+    if lse is not None:
+        _need(lse, torch.float32, "lse")
+    B, Nq, Hq, D = q.shape
+    Hkv, page_size = kpages.shape[1], kpages.shape[2]
+    max_pages = block_table.shape[1]
+    _check(lib().cowa_decode_paged(_ptr(q), _ptr(kpages), _ptr(vpages), _ptr(block_table), _ptr(lens), _ptr(o),
+                                   _ptr(lse) if lse is not None else None, B, Nq, max_pages, page_size, Hq, Hkv, D,
+                                   C.byref(params), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                   _stream()), "cowa_decode_paged")
 
 
 def cowa_decode_static(q, kcache, vcache, lens, o, lse, params):

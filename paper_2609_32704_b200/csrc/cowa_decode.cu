@@ -60,6 +60,11 @@ struct DecodeArgs {
   int B, Tmax, Hq, Hkv, S;
   int sink, near, hkv_global, hkv_offset, full_attn;
   float scale_log2;
+  // extended kernel only: several newest tokens per sequence and / or a paged cache
+  const int32_t* block_table;  // [B, max_pages] page of every page_size-row stretch of a sequence, or nullptr
+  int NQ;                      // query tokens per sequence, at key positions lens[b] - NQ .. lens[b] - 1
+  int tpg, ngroups;            // tokens per block (columns = tpg * Hq / Hkv <= 8), blocks per (sequence, KV head)
+  int page_size, max_pages;
 };
 
 // Position of the v-th visible row (v in the concatenation of the head's ranges).
@@ -87,7 +92,10 @@ __device__ __forceinline__ uint4 ldg128(const void* p) {
   return r;
 }
 
-template <int D, int G>
+// G = columns of the mma n-tile in use.  Plain kernel (EXT = false): the G query heads of the group, one
+// token.  Extended kernel: (token, head) pairs of up to a.tpg of the a.NQ newest tokens, token-major; every
+// column masks the keys its own token must not see; rows may come from a paged cache.
+template <int D, int G, bool EXT>
 // 5 blocks per SM (up to 102 registers, no spills) measured best: fewer, longer splits than at 7 per SM
 __global__ void __launch_bounds__(kThreads, 5) cowa_decode_split_kernel(const DecodeArgs a) {
   static_assert(D == 64 || D == 128, "head dim");
@@ -97,7 +105,8 @@ __global__ void __launch_bounds__(kThreads, 5) cowa_decode_split_kernel(const De
   __shared__ __align__(16) float sc[G * kScStride];  // scores, later the value-phase reduction buffer
   __shared__ float m_s[G], l_s[G];
 
-  const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
+  const int split = blockIdx.x, hk = blockIdx.y;
+  const int b = EXT ? blockIdx.z / a.ngroups : blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int Nk = a.lens[b];
 
@@ -106,7 +115,28 @@ __global__ void __launch_bounds__(kThreads, 5) cowa_decode_split_kernel(const De
   if (a.full_attn) { w.s = 0; w.n = Nk; w.g = 0; w.l = 0; }
   else w = cowa_default_window(Nk, a.hkv_global, a.hkv_offset + hk, a.sink, a.near);
   CowaRange rg[3];
-  const int nr = cowa_decode_ranges(w, Nk, rg);
+  // extended: this block's tokens tq0 .. tq1 sit at key positions Nk - NQ + tq
+  const int gsz = EXT ? a.Hq / a.Hkv : G;
+  const int tq0 = EXT ? (blockIdx.z % a.ngroups) * a.tpg : 0;
+  const int tq1 = EXT ? min(tq0 + a.tpg, a.NQ) - 1 : 0;
+  const int pos0 = EXT ? Nk - a.NQ : Nk - 1;  // key position of token 0
+  const int nr = EXT ? cowa_decode_ranges_span(w, pos0 + tq0, pos0 + tq1, rg) : cowa_decode_ranges(w, Nk, rg);
+  // index of column c in q, o, lse and the split states ([B, NQ, Hq] order)
+  auto col = [&](int c) -> size_t {
+    if constexpr (EXT) return ((size_t)b * a.NQ + tq0 + c / gsz) * a.Hq + (size_t)hk * gsz + c % gsz;
+    else return (size_t)b * a.Hq + (size_t)hk * G + c;
+  };
+  auto col_valid = [&](int c) -> bool { return EXT ? (c < G && tq0 + c / gsz <= tq1) : (c < G); };
+  // address of cache row `tok` of this (sequence, KV head)
+  auto row_ptr = [&](const __nv_bfloat16* base, int tok) -> const __nv_bfloat16* {
+    if constexpr (EXT) {
+      if (a.block_table) {
+        const int pg = a.block_table[(size_t)b * a.max_pages + tok / a.page_size];
+        return base + (((size_t)pg * a.Hkv + hk) * a.page_size + tok % a.page_size) * D;
+      }
+    }
+    return base + ((size_t)b * a.Hkv + hk) * (size_t)a.Tmax * D + (size_t)tok * D;
+  };
   VisMap vm;
   vm.lo0 = rg[0].lo; vm.n0 = nr > 0 ? rg[0].hi - rg[0].lo + 1 : 0;
   vm.lo1 = nr > 1 ? rg[1].lo : 0; vm.n1 = nr > 1 ? rg[1].hi - rg[1].lo + 1 : 0;
@@ -119,19 +149,15 @@ __global__ void __launch_bounds__(kThreads, 5) cowa_decode_split_kernel(const De
   const int c0 = split * chunk;
   const int clen = min(chunk, V - c0);  // <= kChunkCap by the host's choice of S
 
-  const size_t head0 = (size_t)b * a.Hq + (size_t)hk * G;
   if (clen <= 0) {  // empty split: neutral partial state
     for (int i = tid; i < G * D; i += kThreads)
-      a.ws_o[((head0 + i / D) * a.S + split) * D + (i % D)] = 0.f;
-    if (tid < G) {
-      a.ws_m[(head0 + tid) * a.S + split] = -INFINITY;
-      a.ws_l[(head0 + tid) * a.S + split] = 0.f;
+      if (col_valid(i / D)) a.ws_o[(col(i / D) * a.S + split) * D + (i % D)] = 0.f;
+    if (tid < G && col_valid(tid)) {
+      a.ws_m[col(tid) * a.S + split] = -INFINITY;
+      a.ws_l[col(tid) * a.S + split] = 0.f;
     }
     return;
   }
-
-  const __nv_bfloat16* kbase = a.kc + ((size_t)b * a.Hkv + hk) * (size_t)a.Tmax * D;
-  const __nv_bfloat16* vbase = a.vc + ((size_t)b * a.Hkv + hk) * (size_t)a.Tmax * D;
 
   // ---------------- phase 1: scores ----------------
   {
@@ -141,7 +167,7 @@ __global__ void __launch_bounds__(kThreads, 5) cowa_decode_split_kernel(const De
 #pragma unroll
     for (int cc = 0; cc < KC; ++cc) {
       uint4 x = make_uint4(0, 0, 0, 0);
-      if (g < G) x = *reinterpret_cast<const uint4*>(a.q + (head0 + g) * D + cc * 32 + t * 8);
+      if (col_valid(g)) x = *reinterpret_cast<const uint4*>(a.q + col(g) * D + cc * 32 + t * 8);
       bq[cc][0] = x.x; bq[cc][1] = x.y; bq[cc][2] = x.z; bq[cc][3] = x.w;
     }
     const int nblk = (clen + 15) >> 4;
@@ -149,8 +175,8 @@ __global__ void __launch_bounds__(kThreads, 5) cowa_decode_split_kernel(const De
       const int rA = blk * 16 + g, rB = rA + 8;
       const int tokA = vm.token(c0 + min(rA, clen - 1));
       const int tokB = vm.token(c0 + min(rB, clen - 1));
-      const __nv_bfloat16* pa = kbase + (size_t)tokA * D + t * 8;
-      const __nv_bfloat16* pb = kbase + (size_t)tokB * D + t * 8;
+      const __nv_bfloat16* pa = row_ptr(a.kc, tokA) + t * 8;
+      const __nv_bfloat16* pb = row_ptr(a.kc, tokB) + t * 8;
       uint4 ka[KC], kb[KC];
 #pragma unroll
       for (int cc = 0; cc < KC; ++cc) { ka[cc] = ldg128(pa + cc * 32); kb[cc] = ldg128(pb + cc * 32); }
@@ -162,6 +188,13 @@ __global__ void __launch_bounds__(kThreads, 5) cowa_decode_split_kernel(const De
       }
       // c[0],c[1]: row rA, heads 2t, 2t+1;  c[2],c[3]: row rB
       const int h0 = 2 * t, h1 = 2 * t + 1;
+      if constexpr (EXT) {  // a column only sees what its own token sees (Eq. fwa_support at that token's distance)
+        const int p0_ = pos0 + tq0 + h0 / gsz, p1_ = pos0 + tq0 + h1 / gsz;
+        if (!col_valid(h0) || !cowa_visible(w, p0_ - tokA, tokA)) c[0] = -INFINITY;
+        if (!col_valid(h1) || !cowa_visible(w, p1_ - tokA, tokA)) c[1] = -INFINITY;
+        if (!col_valid(h0) || !cowa_visible(w, p0_ - tokB, tokB)) c[2] = -INFINITY;
+        if (!col_valid(h1) || !cowa_visible(w, p1_ - tokB, tokB)) c[3] = -INFINITY;
+      }
       if (rA < clen) {
         if (h0 < G) sc[h0 * kScStride + rA] = c[0] * a.scale_log2;
         if (h1 < G) sc[h1 * kScStride + rA] = c[1] * a.scale_log2;
@@ -182,8 +215,9 @@ __global__ void __launch_bounds__(kThreads, 5) cowa_decode_split_kernel(const De
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
     float l = 0.f;
+    const float msub = (EXT && m == -INFINITY) ? 0.f : m;  // a token that sees none of this split's rows
     for (int r = lane; r < clen; r += 32) {
-      float p = exp2f(s[r] - m);
+      float p = exp2f(s[r] - msub);
       s[r] = p;
       l += p;
     }
@@ -215,7 +249,7 @@ __global__ void __launch_bounds__(kThreads, 5) cowa_decode_split_kernel(const De
       uint4 vv[4][NB];
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
-        const __nv_bfloat16* src = vbase + (size_t)vm.token(c0 + min(rr[k], clen - 1)) * D + g * 8;
+        const __nv_bfloat16* src = row_ptr(a.vc, vm.token(c0 + min(rr[k], clen - 1))) + g * 8;
 #pragma unroll
         for (int bb = 0; bb < NB; ++bb) vv[k][bb] = ldg128(src + bb * 64);
       }
@@ -254,11 +288,11 @@ __global__ void __launch_bounds__(kThreads, 5) cowa_decode_split_kernel(const De
     float s = 0.f;
 #pragma unroll
     for (int r = 0; r < kThreads / 32; ++r) s += sc[r * G * D + i];
-    a.ws_o[((head0 + i / D) * a.S + split) * D + (i % D)] = s;
+    if (col_valid(i / D)) a.ws_o[(col(i / D) * a.S + split) * D + (i % D)] = s;
   }
-  if (tid < G) {
-    a.ws_m[(head0 + tid) * a.S + split] = m_s[tid];
-    a.ws_l[(head0 + tid) * a.S + split] = l_s[tid];
+  if (tid < G && col_valid(tid)) {
+    a.ws_m[col(tid) * a.S + split] = m_s[tid];
+    a.ws_l[col(tid) * a.S + split] = l_s[tid];
   }
 }
 
@@ -353,43 +387,42 @@ int max_visible(int Tmax, int hg, const cowa_params_t* p) {
 
 // Blocks of the split kernel that fit the current device at once (SM count x resident blocks per SM).
 // Falls back to 148 x 5 (B200, up to 102 registers per thread) when no device can be queried.
-template <int D, int G>
+template <int D, int G, bool EXT>
 int resident_blocks_of() {
   int dev = 0, sms = 0, occ = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return 0;
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, cowa_decode_split_kernel<D, G>, kThreads, 0) != cudaSuccess)
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, cowa_decode_split_kernel<D, G, EXT>, kThreads, 0) !=
+      cudaSuccess)
     return 0;
   return sms * occ;
 }
 
+template <bool EXT>
 int resident_blocks(int D, int G) {
   static int cache[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};
   const int di = D == 128 ? 1 : 0, gi = G == 1 ? 0 : G == 2 ? 1 : G == 4 ? 2 : 3;
   if (cache[di][gi] == 0) {
     int r = 0;
-    if (D == 128) r = G == 1 ? resident_blocks_of<128, 1>() : G == 2 ? resident_blocks_of<128, 2>()
-                    : G == 4 ? resident_blocks_of<128, 4>() : resident_blocks_of<128, 8>();
-    else r = G == 1 ? resident_blocks_of<64, 1>() : G == 2 ? resident_blocks_of<64, 2>()
-             : G == 4 ? resident_blocks_of<64, 4>() : resident_blocks_of<64, 8>();
+    if (D == 128) r = G == 1 ? resident_blocks_of<128, 1, EXT>() : G == 2 ? resident_blocks_of<128, 2, EXT>()
+                    : G == 4 ? resident_blocks_of<128, 4, EXT>() : resident_blocks_of<128, 8, EXT>();
+    else r = G == 1 ? resident_blocks_of<64, 1, EXT>() : G == 2 ? resident_blocks_of<64, 2, EXT>()
+             : G == 4 ? resident_blocks_of<64, 4, EXT>() : resident_blocks_of<64, 8, EXT>();
     if (r <= 0) { cudaGetLastError(); return 148 * 5; }
     cache[di][gi] = r;
   }
   return cache[di][gi];
 }
 
-// Splits per (sequence, KV head): the grid should be a whole number of waves of resident blocks, each
-// split at most kChunkCap rows (its scores live in shared memory) and not much shorter than 128 rows.
-int pick_splits(int B, int Tmax, int Hq, int Hkv, int D, const cowa_params_t* p) {
-  const int hg = p->hkv_global > 0 ? p->hkv_global : Hkv;
-  const int vmax = max_visible(Tmax, hg, p);
-  const int heads = B * Hkv;
+// Splits per (sequence, KV head[, token group]): the grid should be a whole number of waves of resident
+// blocks, each split at most kChunkCap rows (its scores live in shared memory) and not much shorter than
+// 128 rows.  `vmax` bounds the visible rows of a block, `units` counts the blocks per split index.
+int splits_for(int vmax, int units, int slots) {
   const int by_cap = (vmax + (kChunkCap - 16) - 1) / (kChunkCap - 16);
   const int by_len = (vmax + 127) / 128;
-  const int slots = resident_blocks(D, Hq / Hkv);
   int s = by_cap;
   for (int waves = 1; waves <= 64; ++waves) {
-    s = (int)(((long long)waves * slots) / heads);
+    s = (int)(((long long)waves * slots) / units);
     if (s >= by_cap && s >= 1) break;
   }
   if (s > by_len) s = by_len;
@@ -397,20 +430,41 @@ int pick_splits(int B, int Tmax, int Hq, int Hkv, int D, const cowa_params_t* p)
   return s < 1 ? 1 : s;
 }
 
-template <int D, int G>
+int pick_splits(int B, int Tmax, int Hq, int Hkv, int D, const cowa_params_t* p) {
+  const int hg = p->hkv_global > 0 ? p->hkv_global : Hkv;
+  return splits_for(max_visible(Tmax, hg, p), B * Hkv, resident_blocks<false>(D, Hq / Hkv));
+}
+
+// Extended kernel: tokens per block and blocks per (sequence, KV head) for NQ tokens and group size gsz.
+void token_groups(int NQ, int gsz, int* tpg, int* ngroups, int* cols) {
+  int t = 1;
+  while (t * 2 * gsz <= 8 && t < NQ) t *= 2;
+  *tpg = t; *ngroups = (NQ + t - 1) / t; *cols = t * gsz;
+}
+
+int pick_splits_ext(int B, int NQ, int Tmax, int Hq, int Hkv, int D, const cowa_params_t* p) {
+  const int hg = p->hkv_global > 0 ? p->hkv_global : Hkv;
+  int tpg, ngroups, cols;
+  token_groups(NQ, Hq / Hkv, &tpg, &ngroups, &cols);
+  long long vmax = (long long)max_visible(Tmax, hg, p) + 3ll * (tpg - 1);  // each range grows by the token span
+  if (vmax > Tmax) vmax = Tmax;
+  return splits_for((int)vmax, B * Hkv * ngroups, resident_blocks<true>(D, cols));
+}
+
+template <int D, int G, bool EXT>
 cudaError_t launch_split(const DecodeArgs& a, cudaStream_t st) {
-  dim3 grid(a.S, a.Hkv, a.B);
-  cowa_decode_split_kernel<D, G><<<grid, kThreads, 0, st>>>(a);
+  dim3 grid(a.S, a.Hkv, EXT ? a.B * a.ngroups : a.B);
+  cowa_decode_split_kernel<D, G, EXT><<<grid, kThreads, 0, st>>>(a);
   return cudaGetLastError();
 }
 
-template <int D>
+template <int D, bool EXT>
 cudaError_t dispatch_split(int G, const DecodeArgs& a, cudaStream_t st) {
   switch (G) {
-    case 1: return launch_split<D, 1>(a, st);
-    case 2: return launch_split<D, 2>(a, st);
-    case 4: return launch_split<D, 4>(a, st);
-    case 8: return launch_split<D, 8>(a, st);
+    case 1: return launch_split<D, 1, EXT>(a, st);
+    case 2: return launch_split<D, 2, EXT>(a, st);
+    case 4: return launch_split<D, 4, EXT>(a, st);
+    case 8: return launch_split<D, 8, EXT>(a, st);
     default: return cudaErrorInvalidValue;
   }
 }
@@ -458,8 +512,9 @@ int decode_launch(const void* q, const void* kc, const void* vc, const int32_t* 
   a.hkv_offset = p->hkv_offset;
   a.full_attn = p->full_attn;
   a.scale_log2 = p->softmax_scale * 1.4426950408889634f;
+  a.block_table = nullptr; a.NQ = 1; a.tpg = 1; a.ngroups = 1; a.page_size = 0; a.max_pages = 0;
   const int G = Hq / Hkv;
-  cudaError_t e = (D == 128) ? dispatch_split<128>(G, a, st) : dispatch_split<64>(G, a, st);
+  cudaError_t e = (D == 128) ? dispatch_split<128, false>(G, a, st) : dispatch_split<64, false>(G, a, st);
   if (e != cudaSuccess) return record_cuda_error(e);
   if (D == 128)
     cowa_decode_combine_kernel<128><<<B * Hq, 128, 0, st>>>(a.ws_o, a.ws_m, a.ws_l,
@@ -472,9 +527,82 @@ int decode_launch(const void* q, const void* kc, const void* vc, const int32_t* 
   return COWA_OK;
 }
 
+// Multi-token and / or paged decode: q, o [B, NQ, Hq, D], lse [B, NQ, Hq]; block_table == nullptr means a
+// contiguous cache [B, Hkv, Tmax, D], otherwise pages [num_pages, Hkv, page_size, D] and Tmax = max_pages * page_size.
+int decode_ext_launch(const void* q, const void* kc, const void* vc, const int32_t* block_table, const int32_t* lens,
+                      void* o, float* lse, int B, int NQ, int Tmax, int page_size, int max_pages, int Hq, int Hkv,
+                      int D, const cowa_params_t* p, int S, void* ws, cudaStream_t st) {
+  DecodeArgs a;
+  a.q = static_cast<const __nv_bfloat16*>(q);
+  a.kc = static_cast<const __nv_bfloat16*>(kc);
+  a.vc = static_cast<const __nv_bfloat16*>(vc);
+  a.lens = lens;
+  const size_t rows = (size_t)B * NQ * Hq;
+  a.ws_o = static_cast<float*>(ws);
+  a.ws_m = a.ws_o + rows * S * D;
+  a.ws_l = a.ws_m + rows * S;
+  a.B = B; a.Tmax = Tmax; a.Hq = Hq; a.Hkv = Hkv; a.S = S;
+  a.sink = p->sink; a.near = p->local;
+  a.hkv_global = p->hkv_global > 0 ? p->hkv_global : Hkv;
+  a.hkv_offset = p->hkv_offset;
+  a.full_attn = p->full_attn;
+  a.scale_log2 = p->softmax_scale * 1.4426950408889634f;
+  a.block_table = block_table; a.NQ = NQ; a.page_size = page_size; a.max_pages = max_pages;
+  int cols;
+  token_groups(NQ, Hq / Hkv, &a.tpg, &a.ngroups, &cols);
+  cudaError_t e = (D == 128) ? dispatch_split<128, true>(cols, a, st) : dispatch_split<64, true>(cols, a, st);
+  if (e != cudaSuccess) return record_cuda_error(e);
+  if (D == 128)
+    cowa_decode_combine_kernel<128><<<(unsigned)rows, 128, 0, st>>>(a.ws_o, a.ws_m, a.ws_l,
+                                                                    static_cast<__nv_bfloat16*>(o), lse, S);
+  else
+    cowa_decode_combine_kernel<64><<<(unsigned)rows, 128, 0, st>>>(a.ws_o, a.ws_m, a.ws_l,
+                                                                   static_cast<__nv_bfloat16*>(o), lse, S);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return record_cuda_error(e);
+  return COWA_OK;
+}
+
 }  // namespace cowa
 
 extern "C" {
+
+size_t cowa_decode_multi_workspace_bytes(int B, int Nq, int Tmax, int Hq, int Hkv, int D, const cowa_params_t* p) {
+  if (!p || B <= 0 || Nq <= 0 || Tmax <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || (D != 64 && D != 128)) return 0;
+  return cowa::decode_ws_bytes(B * Nq, Hq, D, pick_splits_ext(B, Nq, Tmax, Hq, Hkv, D, p));
+}
+
+static int decode_ext(const void* q, const void* kc, const void* vc, const int32_t* block_table, const int32_t* lens,
+                      void* o, float* lse, int B, int Nq, int Tmax, int page_size, int max_pages, int Hq, int Hkv,
+                      int D, const cowa_params_t* p, void* workspace, size_t workspace_bytes, void* stream) {
+  int S = 0;
+  int st = cowa::decode_validate(q, kc, vc, lens, o, B, Tmax, Hq, Hkv, D, p, &S);
+  if (st != COWA_OK) return st;
+  if (Nq <= 0 || Nq > 64 || !workspace) return COWA_ERR_INVALID_ARG;
+  if ((long long)B * ((Nq + 7) / 8 * 8) > 65535) return COWA_ERR_UNSUPPORTED;
+  if (!cowa::aligned16(workspace)) return COWA_ERR_MISALIGNED;
+  S = pick_splits_ext(B, Nq, Tmax, Hq, Hkv, D, p);
+  if (workspace_bytes < cowa::decode_ws_bytes(B * Nq, Hq, D, S)) return COWA_ERR_WORKSPACE_TOO_SMALL;
+  return cowa::decode_ext_launch(q, kc, vc, block_table, lens, o, lse, B, Nq, Tmax, page_size, max_pages, Hq, Hkv, D,
+                                 p, S, workspace, static_cast<cudaStream_t>(stream));
+}
+
+int cowa_decode_multi(const void* q, const void* kcache, const void* vcache, const int32_t* lens, void* o,
+                      float* lse, int B, int Nq, int Tmax, int Hq, int Hkv, int D, const cowa_params_t* p,
+                      void* workspace, size_t workspace_bytes, void* stream) {
+  return decode_ext(q, kcache, vcache, nullptr, lens, o, lse, B, Nq, Tmax, 0, 0, Hq, Hkv, D, p, workspace,
+                    workspace_bytes, stream);
+}
+
+int cowa_decode_paged(const void* q, const void* kpages, const void* vpages, const int32_t* block_table,
+                      const int32_t* lens, void* o, float* lse, int B, int Nq, int max_pages, int page_size,
+                      int Hq, int Hkv, int D, const cowa_params_t* p, void* workspace, size_t workspace_bytes,
+                      void* stream) {
+  if (!block_table || max_pages <= 0 || page_size <= 0 || page_size % 16 != 0) return COWA_ERR_INVALID_ARG;
+  if ((long long)max_pages * page_size > 0x7FFFFFFFll) return COWA_ERR_UNSUPPORTED;
+  return decode_ext(q, kpages, vpages, block_table, lens, o, lse, B, Nq, max_pages * page_size, page_size, max_pages,
+                    Hq, Hkv, D, p, workspace, workspace_bytes, stream);
+}
 
 size_t cowa_decode_workspace_bytes(int B, int Tmax, int Hq, int Hkv, int D, const cowa_params_t* p) {
   if (!p || B <= 0 || Tmax <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || (D != 64 && D != 128)) return 0;

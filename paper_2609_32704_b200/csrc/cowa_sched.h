@@ -184,3 +184,27 @@ COWA_HD int cowa_decode_ranges(const CowaWin& w, int Nk, CowaRange out[3]) {
   }
   return n;
 }
+
+// Several queries at once (multi-token decode): queries at key positions p0 .. p1 (p1 = Nk - 1 for the
+// newest token); the union of their visible keys, same form as cowa_decode_ranges.  Which query sees
+// which key inside the union is decided per element with cowa_visible.
+COWA_HD int cowa_decode_ranges_span(const CowaWin& w, int p0, int p1, CowaRange out[3]) {
+  CowaRange c[3];
+  int nc = 0;
+  if (w.s > 0) { c[nc].lo = 0; c[nc].hi = cowa_imin(w.s - 1, p1); nc++; }
+  if (w.l > 0) {
+    long long lo = (long long)p0 - w.n - w.g - w.l + 1, hi = (long long)p1 - w.n - w.g;
+    if (lo < 0) lo = 0;
+    if (hi >= lo) { c[nc].lo = (int)lo; c[nc].hi = (int)hi; nc++; }
+  }
+  if (w.n > 0) { c[nc].lo = cowa_imax(p0 - w.n + 1, 0); c[nc].hi = p1; nc++; }
+  int n = 0;
+  for (int i = 0; i < nc; ++i) {
+    if (n > 0 && c[i].lo <= out[n - 1].hi + 1) {
+      out[n - 1].hi = cowa_imax(out[n - 1].hi, c[i].hi);
+    } else {
+      out[n++] = c[i];
+    }
+  }
+  return n;
+}

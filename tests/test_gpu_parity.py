@@ -529,3 +529,99 @@ def test_decode_equals_last_forward_row():
     o_d, lse_d = run_decode(q[:, :, T - 1].contiguous(), k, v, lens, params)
     assert (o_d.float() - o_f[:, :, T - 1].float()).abs().max().item() <= 2e-2
     assert (lse_d - lse_f[:, :, T - 1]).abs().max().item() <= 1e-3
+
+
+# ------------------------------------------------------------------ multi-token and paged decode
+
+def multi_case(B, Nq, Tmax, Hq, Hkv, D, sink, local, lens, page_size=None, full_attn=False, seed=62):
+    """The Nq newest tokens of every sequence against the oracle's forward with N_q = Nq, N_k = lens[b]."""
+    q = cowa_inputs.make_train_inputs(seed, B, Nq, Hq, Hkv, D)[0].permute(0, 2, 1, 3).contiguous()  # [B,Nq,Hq,D]
+    _, kc, vc, _ = cowa_inputs.make_decode_inputs(seed + 1, B, Tmax, Hq, Hkv, D, Tmax, Tmax)
+    lens_t = torch.tensor(lens, dtype=torch.int32)
+    for b in range(B):
+        kc[b, :, lens[b]:] = float("nan")
+        vc[b, :, lens[b]:] = float("nan")
+    scale = cowa_inputs.softmax_scale(D)
+    params = cowa.make_params(sink=sink, local=local, softmax_scale=scale, full_attn=full_attn)
+    o = torch.full_like(q, float("nan")).to(DEV)
+    lse = torch.full((B, Nq, Hq), float("nan"), dtype=torch.float32, device=DEV)
+    if page_size is None:
+        nbytes = cowa.cowa_decode_multi_workspace_bytes(B, Nq, Tmax, Hq, Hkv, D, params)
+        ws = torch.empty(nbytes + 64, dtype=torch.uint8, device=DEV)
+        ws.fill_(0xFF)
+        cowa.cowa_decode_multi(q.to(DEV), kc.to(DEV), vc.to(DEV), lens_t.to(DEV), o, lse, params, ws[:nbytes])
+    else:
+        max_pages = (Tmax + page_size - 1) // page_size
+        num_pages = B * max_pages + 5
+        g = torch.Generator().manual_seed(seed)
+        perm = torch.randperm(num_pages, generator=g)
+        table = torch.full((B, max_pages), -1, dtype=torch.int32)
+        kp = torch.full((num_pages, Hkv, page_size, D), float("nan"), dtype=torch.bfloat16)
+        vp = torch.full_like(kp, float("nan"))
+        n = 0
+        for b in range(B):
+            for i in range((lens[b] + page_size - 1) // page_size):  # pages past the sequence stay unmapped
+                pg = int(perm[n]); n += 1
+                table[b, i] = pg
+                rows = min(page_size, Tmax - i * page_size)
+                kp[pg, :, :rows] = kc[b, :, i * page_size:i * page_size + rows]
+                vp[pg, :, :rows] = vc[b, :, i * page_size:i * page_size + rows]
+        nbytes = cowa.cowa_decode_multi_workspace_bytes(B, Nq, max_pages * page_size, Hq, Hkv, D, params)
+        ws = torch.empty(nbytes + 64, dtype=torch.uint8, device=DEV)
+        ws.fill_(0xFF)
+        cowa.cowa_decode_paged(q.to(DEV), kp.to(DEV), vp.to(DEV), table.to(DEV), lens_t.to(DEV), o, lse, params,
+                               ws[:nbytes])
+    torch.cuda.synchronize()
+    cowa.cowa_check_device_status()
+    assert (ws[nbytes:] == 0xFF).all(), "decode wrote past its workspace"
+    f = cowa_inputs.to_f64
+    for b in range(B):
+        n = lens[b]
+        ws_ = [(0, n, 0, 0)] * Hkv if full_attn else orc.default_windows(n, Hkv, sink, local)
+        o_ref, lse_ref = orc.forward(f(q[b].permute(1, 0, 2)), f(kc[b, :, :n]), f(vc[b, :, :n]), ws_, scale)
+        check(f"multi lse[b={b}]", lse[b].permute(1, 0).cpu().numpy(), lse_ref, TOL_LSE, TOL_LSE)
+        check(f"multi o[b={b}]", o[b].permute(1, 0, 2).float().cpu().numpy(), o_ref)
+
+
+@pytest.mark.parametrize("B,Nq,Tmax,Hq,Hkv,D,sink,local,lens", [
+    (2, 2, 5000, 8, 2, 128, 16, 100, [5000, 2777]),        # G = 4: both tokens share one pass
+    (2, 5, 3000, 8, 2, 128, 16, 100, [3000, 5]),           # three token groups, the last half empty; len = Nq
+    (2, 8, 3001, 4, 4, 64, 4, 31, [3001, 17]),             # G = 1: eight tokens in one pass, D = 64
+    (1, 3, 4096, 16, 2, 128, 128, 512, [4096]),            # G = 8: one token per block
+    (3, 3, 2000, 4, 2, 128, 7, 50, [2000, 640, 57]),       # G = 2, odd token count; a dense short sequence
+    (1, 4, 40000, 4, 2, 128, 128, 4096, [39999]),          # several splits per head
+    (1, 1, 2500, 8, 2, 128, 16, 100, [2400]),              # Nq = 1 through the extended kernel
+])
+def test_decode_multi_shapes(B, Nq, Tmax, Hq, Hkv, D, sink, local, lens):
+    multi_case(B, Nq, Tmax, Hq, Hkv, D, sink, local, lens)
+
+
+def test_decode_multi_full_attn():
+    multi_case(2, 4, 6000, 8, 2, 128, 0, 1, [6000, 4321], full_attn=True)
+
+
+@pytest.mark.parametrize("B,Nq,Tmax,Hq,Hkv,D,sink,local,lens,page", [
+    (3, 1, 5000, 8, 2, 128, 16, 100, [5000, 1, 2777], 16),
+    (2, 4, 4100, 8, 4, 128, 32, 200, [4100, 999], 64),
+    (2, 2, 8192, 16, 2, 64, 128, 512, [8192, 640], 256),
+    (1, 1, 40000, 4, 2, 128, 128, 4096, [39999], 128),
+])
+def test_decode_paged_shapes(B, Nq, Tmax, Hq, Hkv, D, sink, local, lens, page):
+    multi_case(B, Nq, Tmax, Hq, Hkv, D, sink, local, lens, page_size=page)
+
+
+def test_decode_multi_last_token_equals_single_token_decode():
+    # the newest of the Nq tokens is the token cowa_decode computes for the same cache
+    B, Nq, Tmax, Hq, Hkv, D = 2, 4, 3000, 8, 2, 128
+    q = cowa_inputs.make_train_inputs(64, B, Nq, Hq, Hkv, D, device=DEV)[0].permute(0, 2, 1, 3).contiguous()
+    _, kc, vc, _ = cowa_inputs.make_decode_inputs(65, B, Tmax, Hq, Hkv, D, Tmax, Tmax, device=DEV)
+    lens = torch.tensor([3000, 1234], dtype=torch.int32, device=DEV)
+    params = cowa.make_params(sink=16, local=128, softmax_scale=cowa_inputs.softmax_scale(D))
+    o = torch.empty_like(q)
+    lse = torch.empty((B, Nq, Hq), dtype=torch.float32, device=DEV)
+    ws = torch.empty(cowa.cowa_decode_multi_workspace_bytes(B, Nq, Tmax, Hq, Hkv, D, params), dtype=torch.uint8,
+                     device=DEV)
+    cowa.cowa_decode_multi(q, kc, vc, lens, o, lse, params, ws)
+    o1, lse1 = run_decode(q[:, Nq - 1].contiguous(), kc, vc, lens, params)
+    assert (o[:, Nq - 1].float() - o1.float()).abs().max().item() <= 1e-2
+    assert (lse[:, Nq - 1] - lse1).abs().max().item() <= 1e-4
