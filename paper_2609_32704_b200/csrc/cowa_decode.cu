@@ -105,6 +105,9 @@ __global__ void __launch_bounds__(kThreads, 5) cowa_decode_split_kernel(const De
   __shared__ __align__(16) float sc[G * kScStride];  // scores, later the value-phase reduction buffer
   __shared__ float m_s[G], l_s[G];
 
+  // The merge kernel is launched with programmatic stream serialisation: once every block of this grid has
+  // started, its blocks may be scheduled and wait (griddepcontrol.wait) for this grid's results.
+  asm volatile("griddepcontrol.launch_dependents;");
   const int split = blockIdx.x, hk = blockIdx.y;
   const int b = EXT ? blockIdx.z / a.ngroups : blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -310,6 +313,7 @@ __global__ void __launch_bounds__(128) cowa_decode_combine_kernel(const float* _
   __shared__ float part[4][D];
   const size_t bh = blockIdx.x;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // the split kernel's states are complete and visible
   const float* m = ws_m + bh * S;
   const float* l = ws_l + bh * S;
   const float* po = ws_o + bh * S * D + lane * V;
@@ -451,6 +455,19 @@ int pick_splits_ext(int B, int NQ, int Tmax, int Hq, int Hkv, int D, const cowa_
   return splits_for((int)vmax, B * Hkv * ngroups, resident_blocks<true>(D, cols));
 }
 
+// Launch of the merge kernel right behind the split kernel, allowed to start before that one has drained.
+template <int D>
+cudaError_t launch_combine(unsigned rows, const float* ws_o, const float* ws_m, const float* ws_l, __nv_bfloat16* o,
+                           float* lse, int S, cudaStream_t st) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(rows); cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, cowa_decode_combine_kernel<D>, ws_o, ws_m, ws_l, o, lse, S);
+}
+
 template <int D, int G, bool EXT>
 cudaError_t launch_split(const DecodeArgs& a, cudaStream_t st) {
   dim3 grid(a.S, a.Hkv, EXT ? a.B * a.ngroups : a.B);
@@ -516,13 +533,8 @@ int decode_launch(const void* q, const void* kc, const void* vc, const int32_t* 
   const int G = Hq / Hkv;
   cudaError_t e = (D == 128) ? dispatch_split<128, false>(G, a, st) : dispatch_split<64, false>(G, a, st);
   if (e != cudaSuccess) return record_cuda_error(e);
-  if (D == 128)
-    cowa_decode_combine_kernel<128><<<B * Hq, 128, 0, st>>>(a.ws_o, a.ws_m, a.ws_l,
-                                                            static_cast<__nv_bfloat16*>(o), lse, S);
-  else
-    cowa_decode_combine_kernel<64><<<B * Hq, 128, 0, st>>>(a.ws_o, a.ws_m, a.ws_l,
-                                                          static_cast<__nv_bfloat16*>(o), lse, S);
-  e = cudaGetLastError();
+  e = (D == 128) ? launch_combine<128>((unsigned)(B * Hq), a.ws_o, a.ws_m, a.ws_l, static_cast<__nv_bfloat16*>(o), lse, S, st)
+                 : launch_combine<64>((unsigned)(B * Hq), a.ws_o, a.ws_m, a.ws_l, static_cast<__nv_bfloat16*>(o), lse, S, st);
   if (e != cudaSuccess) return record_cuda_error(e);
   return COWA_OK;
 }
@@ -552,13 +564,8 @@ int decode_ext_launch(const void* q, const void* kc, const void* vc, const int32
   token_groups(NQ, Hq / Hkv, &a.tpg, &a.ngroups, &cols);
   cudaError_t e = (D == 128) ? dispatch_split<128, true>(cols, a, st) : dispatch_split<64, true>(cols, a, st);
   if (e != cudaSuccess) return record_cuda_error(e);
-  if (D == 128)
-    cowa_decode_combine_kernel<128><<<(unsigned)rows, 128, 0, st>>>(a.ws_o, a.ws_m, a.ws_l,
-                                                                    static_cast<__nv_bfloat16*>(o), lse, S);
-  else
-    cowa_decode_combine_kernel<64><<<(unsigned)rows, 128, 0, st>>>(a.ws_o, a.ws_m, a.ws_l,
-                                                                   static_cast<__nv_bfloat16*>(o), lse, S);
-  e = cudaGetLastError();
+  e = (D == 128) ? launch_combine<128>((unsigned)rows, a.ws_o, a.ws_m, a.ws_l, static_cast<__nv_bfloat16*>(o), lse, S, st)
+                 : launch_combine<64>((unsigned)rows, a.ws_o, a.ws_m, a.ws_l, static_cast<__nv_bfloat16*>(o), lse, S, st);
   if (e != cudaSuccess) return record_cuda_error(e);
   return COWA_OK;
 }
