@@ -160,6 +160,28 @@ def oracle_sample(budget_s, seed_tiles=0):
     return flops, secs, units
 
 
+def count_legal_pairs(T, windows):
+    """Legal (query, key) pairs summed over the KV heads for N_q = N_k = T (accounting only: the
+    second FLOP figure beside the visited-tile one).  Per query row the sink, band and near
+    intervals of keys are clipped to the causal prefix and their union is measured."""
+    import numpy as np
+    iq = np.arange(T, dtype=np.int64)
+    total = 0
+    for s_, n_, g_, l_ in windows:
+        near_lo = np.maximum(iq - n_ + 1, 0)                      # near: [near_lo, iq]
+        band_lo = np.maximum(iq - (n_ + g_ + l_) + 1, 0)          # band: [band_lo, band_hi]
+        band_hi = iq - (n_ + g_)
+        band = np.where(l_ > 0, np.maximum(band_hi - band_lo + 1, 0), 0)
+        sink_hi = np.minimum(s_ - 1, iq)                          # sink: [0, sink_hi]
+        # the three intervals are ordered sink <= band <= near; subtract the overlaps of neighbours
+        sink = np.maximum(sink_hi + 1, 0)
+        top_of_lower = np.where(band > 0, band_hi, -1)
+        near = iq - np.maximum(near_lo, np.maximum(top_of_lower, sink_hi) + 1) + 1
+        band_eff = np.where(band > 0, np.maximum(band_hi - np.maximum(band_lo, sink_hi + 1) + 1, 0), 0)
+        total += int(sink.sum() + band_eff.sum() + np.maximum(near, 0).sum())
+    return total
+
+
 def cpu_threads():
     try:
         from threadpoolctl import threadpool_info
@@ -242,6 +264,7 @@ def run_cuda(args):
     cnt = cowa.cowa_tile_counts(T, T, Hkv, p_train)
     cnt_full = cowa.cowa_tile_counts(T, T, Hkv, p_full)
     G = Hq // Hkv
+    legal_pairs = count_legal_pairs(T, cowa.cowa_default_windows(T, Hkv, 0, Hkv, ct["sink"], ct["local"]))
     fwd_flops = cnt["visited"] * 128 * 128 * 4 * D * G * B
     bwd_flops = 2.5 * fwd_flops
     full_fwd_flops = cnt_full["visited"] * 128 * 128 * 4 * D * G * B
@@ -297,6 +320,9 @@ def run_cuda(args):
     fwd_ms = sum(e[0].elapsed_time(e[1]) for e in evs) / args.steps
     bwd_ms = sum(e[1].elapsed_time(e[2]) for e in evs) / args.steps
     dec_ms = sum(e[2].elapsed_time(e[3]) for e in evs) / args.steps
+    fwd_min = max_over_ranks(min(e[0].elapsed_time(e[1]) for e in evs), world)
+    bwd_min = max_over_ranks(min(e[1].elapsed_time(e[2]) for e in evs), world)
+    dec_min = max_over_ranks(min(e[2].elapsed_time(e[3]) for e in evs), world)
     total_ms = evs[0][0].elapsed_time(evs[-1][3]) / args.steps
     fwd_ms, bwd_ms, dec_ms, total_ms = (max_over_ranks(x, world) for x in (fwd_ms, bwd_ms, dec_ms, total_ms))
 
@@ -516,15 +542,17 @@ def run_cuda(args):
     traffic_128k = {"cowa_bwd_kernel<128>": 12.904e9 + 6.795e9, "cowa_fwd_kernel<128, 0>": 9.546e9 + 1.055e9}
     roofline = {"kernel": dom, "bound": "tensor", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s",
                 "frac": achieved / peak_tf, "peak_source": f"{peak_src} bf16 sustained (kernel timed inside a long step)",
-                "frac_of_burst_peak": achieved / peaks["bf16_tflops"],
+                "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "frac_of_nominal_2250": achieved / 2250.0,
                 "traffic": traffic_128k.get(dom) if args.train_cfg == "128k" else None,
                 "traffic_unit": "bytes per launch (ncu, 128K workload)"}
     dec_gbs = dec_bytes / (dec_ms * 1e-3) / 1e9
     b2b_gbs = dec_bytes / (dec_b2b_ms * 1e-3) / 1e9
     decode = {"us_per_step": dec_ms * 1e3, "us_per_token": dec_ms * 1e3 / cd["B"], "visible_kv_bytes": dec_bytes,
               "achieved_gbs": dec_gbs, "hbm_peak_gbs": peaks["hbm_gbs"], "frac_hbm": dec_gbs / peaks["hbm_gbs"],
+              "frac_nominal_8tbs": dec_gbs / 8000.0, "us_per_step_min": dec_min * 1e3,
               "back_to_back": {"us_per_call": dec_b2b_ms * 1e3, "achieved_gbs": b2b_gbs,
-                               "frac_hbm": b2b_gbs / peaks["hbm_gbs"], "calls": n_dec}}
+                               "frac_hbm": b2b_gbs / peaks["hbm_gbs"], "frac_nominal_8tbs": b2b_gbs / 8000.0,
+                               "calls": n_dec}}
 
     cpu = None
     if not args.no_cpu_baseline:
@@ -542,7 +570,10 @@ def run_cuda(args):
                    "phases": ["fwd"] + (["bwd"] if have_bwd else []) + ["decode"],
                    "l2": "inputs larger than L2 (2.6 GB training tensors, 0.57 GB visible KV cache)",
                    "parallelism": "independent replicas" if world > 1 else "single GPU"},
-        "fwd_ms": fwd_ms, "fwd_tflops": fwd_flops / fwd_ms / 1e9,
+        "fwd_ms": fwd_ms, "fwd_ms_min": fwd_min, "fwd_tflops": fwd_flops / fwd_ms / 1e9,
+        "fwd_tflops_legal_pairs": legal_pairs * 4 * D * G * B / fwd_ms / 1e9,
+        "bwd_ms_min": bwd_min if have_bwd else None,
+        "bwd_tflops_legal_pairs": legal_pairs * 10 * D * G * B / bwd_ms / 1e9 if have_bwd else None,
         "bwd_ms": bwd_ms if have_bwd else None, "bwd_tflops": bwd_flops / bwd_ms / 1e9 if have_bwd else None,
         "bwd_main_kernel_ms": bwd_main_ms,
         "visited_tiles": cnt["visited"], "causal_tiles": cnt["causal"],

@@ -167,6 +167,18 @@ def test_equal_area_schedule_balances_visited_tiles():
     assert abs(sum(eq) - sum(df)) / sum(df) < 0.02   # same total work, redistributed
 
 
+def test_bench_legal_pair_count_matches_masks():
+    import bench
+    rng = np.random.default_rng(7)
+    cases = [(300, 4, 7, 20), (1000, 8, 128, 100), (257, 3, 0, 1), (64, 2, 40, 40)]
+    cases += [(int(rng.integers(1, 700)), int(rng.integers(1, 9)), int(rng.integers(0, 200)), int(rng.integers(1, 300)))
+              for _ in range(20)]
+    for T, H, s_, n_ in cases:
+        ws = cowa.cowa_default_windows(T, H, 0, H, s_, n_)
+        want = sum(int(orc.visible_mask(T, T, w).sum()) for w in ws)
+        assert bench.count_legal_pairs(T, ws) == want, (T, H, s_, n_)
+
+
 def test_decode_schedule():
     for Nk, Hkv, sink, near, Bk in [(131072, 8, 128, 4096, 128), (98304, 8, 128, 4096, 128),
                                     (100001, 8, 128, 4096, 128), (777, 4, 5, 60, 64), (50, 8, 30, 30, 16),
