@@ -448,6 +448,39 @@ def test_128k_config_sampled():
                        kv_samples=[(6, 901)])
 
 
+def test_one_million_tokens_sampled():
+    """Largest size exercised: T = 2^20 (indices and byte offsets beyond 2^31 in the tensors).  Forward
+    and backward run in full; O, LSE and dQ are compared on sampled query tiles, decode on the full row."""
+    T, Hq, Hkv, D, sink, local = 1 << 20, 2, 2, 64, 128, 4096
+    q, k, v, d_o = cowa_inputs.make_train_inputs(77, 1, T, Hq, Hkv, D, device=DEV)
+    scale = cowa_inputs.softmax_scale(D)
+    params = cowa.make_params(sink=sink, local=local, softmax_scale=scale)
+    o, lse = run_fwd(q, k, v, params)
+    dq, dk, dv = (torch.empty_like(x) for x in (q, k, v))
+    ws_b = torch.empty(cowa.cowa_bwd_workspace_bytes(1, T, Hq, Hkv, D, params), dtype=torch.uint8, device=DEV)
+    cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, params, ws_b)
+    torch.cuda.synchronize()
+    cowa.cowa_check_device_status()
+    del ws_b
+    assert torch.isfinite(dk.float()).all() and torch.isfinite(dv.float()).all()
+    ws = orc.default_windows(T, Hkv, sink, local)
+    f = cowa_inputs.to_f64
+    for h, tile in [(0, 0), (1, T // 128 - 1), (0, 5000)]:
+        rows = np.arange(tile * 128, tile * 128 + 128)
+        qh, kh, vh, doh = f(q[0, h:h + 1]), f(k[0, h:h + 1]), f(v[0, h:h + 1]), f(d_o[0, h:h + 1])
+        o_ref, lse_ref = orc.forward_rows(qh, kh, vh, [ws[h]], scale, 0, rows)
+        check(f"1M lse[h{h},tile{tile}]", lse[0, h, rows].cpu().numpy(), lse_ref, TOL_LSE, TOL_LSE)
+        check(f"1M o[h{h},tile{tile}]", o[0, h, rows].float().cpu().numpy(), o_ref)
+        dq_ref = orc.backward_dq_rows(qh, kh, vh, doh, [ws[h]], scale, 0, rows)
+        check_grad(f"1M dq[h{h},tile{tile}]", dq[0, h, rows].float().cpu().numpy(), dq_ref)
+        del qh, kh, vh, doh
+    # decode of the last position on the same tensors used as a cache of length T
+    lens = torch.tensor([T], dtype=torch.int32, device=DEV)
+    o_d, lse_d = run_decode(q[:, :, T - 1].contiguous(), k, v, lens, params)
+    assert (o_d.float() - o[:, :, T - 1].float()).abs().max().item() <= 2e-2
+    assert (lse_d - lse[:, :, T - 1]).abs().max().item() <= 1e-3
+
+
 # ------------------------------------------------------------------ decode
 
 def run_decode(q, kc, vc, lens, params):
