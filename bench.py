@@ -469,7 +469,26 @@ def run_cuda(args):
         cowa.cowa_check_device_status()
         varlen = {"lengths": mix, "ms": times["packed"], "tflops": v_flops / times["packed"] / 1e9,
                   "one_call_per_sequence_ms": times["one_by_one"]}
-        del pq, pk, pv, po, plse, seq_q, seq_k, seq_v, seq_o, seq_l
+        del seq_q, seq_k, seq_v, seq_o, seq_l
+        if have_bwd:  # backward over the same packed batch (N_q = N_k per sequence)
+            pdo = cowa_inputs.make_train_inputs(8, 1, tot, Hq, Hkv, D, device=dev)[3][0]
+            pdq, pdk, pdv = torch.empty_like(pq), torch.empty_like(pk), torch.empty_like(pv)
+            wsv = torch.empty(cowa.cowa_bwd_varlen_workspace_bytes(len(mix), tot, Hq, Hkv, D, p_mix), dtype=torch.uint8,
+                              device=dev)
+            fn = lambda: cowa.cowa_bwd_varlen(pq, pk, pv, po, plse, pdo, pdq, pdk, pdv, cu, p_mix, wsv)
+            for _ in range(2):
+                fn()
+            ev2 = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+            ev2[0].record()
+            for _ in range(3):
+                fn()
+            ev2[1].record()
+            torch.cuda.synchronize()
+            cowa.cowa_check_device_status()
+            b_ms = max_over_ranks(ev2[0].elapsed_time(ev2[1]) / 3, world)
+            varlen.update({"bwd_ms": b_ms, "bwd_tflops": 2.5 * v_flops / b_ms / 1e9})
+            del pdo, pdq, pdk, pdv, wsv
+        del pq, pk, pv, po, plse
 
     # ---- end to end: host buffers in, results back to the host, copies inside the timed region ----
     e2e = None

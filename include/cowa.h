@@ -125,6 +125,20 @@ int cowa_bwd(const void* q, const void* k, const void* v, const void* o, const f
  * on the call's stream (both are cudaEvent_t handles owned by the caller; NULL, NULL switches it off). */
 int cowa_bwd_set_profile_events(void* start_event, void* stop_event);
 
+/* Training backward over a packed batch of B sequences of different lengths (self-attention: N_q = N_k =
+ * the sequence's length; Algorithm 2 applied per sequence, each with windows from its own length, Sec. 2.1).
+ *   q, o, d_o, dq [Hq,total,D]; k, v, dk, dv [Hkv,total,D] bf16; lse [Hq,total] fp32 as written by
+ *   cowa_prefill_varlen for the same offsets with cu_seqlens_q = cu_seqlens_k = cu_seqlens;
+ *   cu_seqlens: DEVICE int32[B+1], cu[0] = 0, cu[B] = total, non-decreasing.
+ * dq, dk, dv are fully overwritten for every row of every sequence.  Malformed offsets are reported as for
+ * cowa_prefill_varlen.  `workspace`: device, >= cowa_bwd_varlen_workspace_bytes(B, total, ...), 16-byte
+ * aligned, no initialisation needed.  cowa_params_t.deterministic applies as in cowa_bwd. */
+int cowa_bwd_varlen(const void* q, const void* k, const void* v, const void* o, const float* lse,
+                    const void* d_o, void* dq, void* dk, void* dv, const int32_t* cu_seqlens,
+                    int B, int total, int Hq, int Hkv, int D, const cowa_params_t* p,
+                    void* workspace, size_t workspace_bytes, void* stream);
+size_t cowa_bwd_varlen_workspace_bytes(int B, int total, int Hq, int Hkv, int D, const cowa_params_t* p);
+
 /* Single-token decode over a KV cache (Sec. 2.3 "Decoding"): the forward with N_q = 1.
  *   q [B,Hq,D]; kcache,vcache [B,Hkv,Tmax,D]; lens int32 [B] on the DEVICE, lens[b] = N_k
  *   = cached tokens + 1, the current token's K/V already stored at index lens[b]-1.

@@ -54,6 +54,10 @@ def lib():
         L.cowa_prefill_varlen.restype = i32
         L.cowa_bwd.argtypes = [vp] * 9 + [i32] * 5 + [pp, vp, sz, vp]
         L.cowa_bwd.restype = i32
+        L.cowa_bwd_varlen.argtypes = [vp] * 10 + [i32] * 5 + [pp, vp, sz, vp]
+        L.cowa_bwd_varlen.restype = i32
+        L.cowa_bwd_varlen_workspace_bytes.argtypes = [i32] * 5 + [pp]
+        L.cowa_bwd_varlen_workspace_bytes.restype = sz
         L.cowa_decode.argtypes = [vp] * 6 + [i32] * 5 + [pp, vp, sz, vp]
         L.cowa_decode.restype = i32
         L.cowa_decode_static.argtypes = [vp] * 6 + [i32] * 5 + [pp, vp]
@@ -186,6 +190,26 @@ def cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, params, workspace):
     _check(lib().cowa_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(d_o), _ptr(dq), _ptr(dk),
                           _ptr(dv), B, T, Hq, Hkv, D, C.byref(params), _ptr(workspace),
                           workspace.numel() * workspace.element_size(), _stream()), "cowa_bwd")
+
+
+def cowa_bwd_varlen_workspace_bytes(B, total, Hq, Hkv, D, params):
+    return int(lib().cowa_bwd_varlen_workspace_bytes(B, total, Hq, Hkv, D, C.byref(params)))
+
+
+def cowa_bwd_varlen(q, k, v, o, lse, d_o, dq, dk, dv, cu_seqlens, params, workspace):
+    """Packed batch (N_q = N_k per sequence): q/o/d_o/dq [Hq,total,D], k/v/dk/dv [Hkv,total,D], lse [Hq,total];
+    cu_seqlens CUDA int32 [B+1]."""
+    import torch
+    for t, n in ((q, "q"), (k, "k"), (v, "v"), (o, "o"), (d_o, "d_o"), (dq, "dq"), (dk, "dk"), (dv, "dv")):
+        _need(t, torch.bfloat16, n)
+    _need(lse, torch.float32, "lse")
+    _need(cu_seqlens, torch.int32, "cu_seqlens")
+    Hq, total, D = q.shape
+    Hkv = k.shape[0]
+    B = cu_seqlens.numel() - 1
+    _check(lib().cowa_bwd_varlen(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(d_o), _ptr(dq), _ptr(dk),
+                                 _ptr(dv), _ptr(cu_seqlens), B, total, Hq, Hkv, D, C.byref(params), _ptr(workspace),
+                                 workspace.numel() * workspace.element_size(), _stream()), "cowa_bwd_varlen")
 
 
 def cowa_bwd_set_profile_events(start_event, stop_event):

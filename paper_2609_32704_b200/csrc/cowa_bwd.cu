@@ -51,6 +51,12 @@ struct BwdArgs {
   int dq_fixed;        // 1: dQ partial sums travel as 32-bit fixed point (order-independent addition)
   int parts;           // blocks per KV tile: each takes G / parts heads of the group (1: the whole group)
   float* dkv_part;     // parts > 1: fp32 partial dK, dV [B*Hkv, nKV, parts, 2, BKV, D], summed by a last kernel
+  // packed (variable-length) batches only: tensors are [H, total, D], sequence b owns rows cu[b] .. cu[b+1]
+  const int* cu;       // [B+1] device
+  __nv_bfloat16* dk;   // raw outputs for the last, partial KV tile of a sequence
+  __nv_bfloat16* dv;
+  int total, tiles_bound;  // rows of the packed tensors; grid tiles per KV head (upper bound of the real count)
+  int sink, local, hkv_global, hkv_offset, full_attn, explicit_windows;
   float scale, scale_log2;
   CowaHeadWindows wins;
 };
@@ -87,7 +93,7 @@ __device__ __forceinline__ uint32_t interval_bits32(long long a, long long b, lo
 // named barrier for one 128-thread warpgroup
 __device__ __forceinline__ void wg_sync(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
 
-template <int D>
+template <int D, bool VARLEN>
 __global__ void __launch_bounds__(512, 1)
 cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmdO,
@@ -129,8 +135,12 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 
   // ---- work item: sink tiles of every head first, then head-major with ascending KV tile ----
   int hk, b, j;
-  const int part = blockIdx.x % a.parts;
-  {
+  const int part = VARLEN ? 0 : blockIdx.x % a.parts;
+  // Sequence geometry.  Packed batches: N_q = N_k = the sequence's length, rows start at cu[b]; the fp32
+  // dQ accumulator and the LSE / Delta vectors are laid out with every sequence padded to 64 rows (pbase).
+  int Nq = a.Nq, Nk = a.Nk, rbase = 0, pbase = 0;
+  CowaWin w;
+  if constexpr (!VARLEN) {
     int idx = blockIdx.x / a.parts;
     const int nKV = (a.Nk + BKV - 1) / BKV, nsk = a.sink_tiles, nhead = a.B * a.Hkv;
     if (idx < nsk * nhead) {
@@ -140,17 +150,33 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       j = nsk + idx % (nKV - nsk); idx /= (nKV - nsk);
     }
     hk = idx % a.Hkv; b = idx / a.Hkv;
+    w = a.wins.w[hk];
+  } else {
+    // head-major: consecutive blocks are consecutive KV tiles of one head (their dQ rows overlap in L2)
+    hk = blockIdx.x / a.tiles_bound;
+    int nts;
+    if (!varlen_locate(a.cu, a.B, blockIdx.x % a.tiles_bound, BKV, BQS, &b, &j, &nts, &pbase)) return;
+    rbase = a.cu[b];
+    Nq = Nk = a.cu[b + 1] - rbase;
+    if (rbase < 0 || rbase + Nk > a.total) {  // malformed offsets: report, touch nothing
+      if (threadIdx.x == 0) atomicOr(a.status, 2u);
+      return;
+    }
+    w = a.wins.w[hk];
+    if (a.full_attn) { w.s = 0; w.n = Nk; w.g = 0; w.l = 0; }
+    else if (!a.explicit_windows) w = cowa_default_window(Nk, a.hkv_global, a.hkv_offset + hk, a.sink, a.local);
   }
-  const int off = a.Nk - a.Nq;
-  const int k0 = j * BKV, k1 = min(k0 + BKV, a.Nk) - 1;
-  const CowaWin w = a.wins.w[hk];
+  const int off = Nk - Nq;
+  const int k0 = j * BKV, k1 = min(k0 + BKV, Nk) - 1;
   CowaRange rg[2];
-  cowa_bwd_ranges(w, k0, k1, off, a.Nq, BQS, rg);
+  cowa_bwd_ranges(w, k0, k1, off, Nq, BQS, rg);
   const int cnt = cowa_range_len(rg[0]) + cowa_range_len(rg[1]);  // QO steps per head
   const int gs = a.G / a.parts;          // heads of the group handled by this block
   const int N = cnt * gs;
-  const int bhk = b * a.Hkv + hk;
-  const int bhq0 = b * a.Hq + hk * a.G + part * gs;  // first of them
+  const int bhk = VARLEN ? hk : b * a.Hkv + hk;                                     // third TMA coordinate of K, V, dK, dV
+  const int bhq0 = (VARLEN ? 0 : b * a.Hq) + hk * a.G + part * gs;                  // ... of Q, dO, dQ: first head of this block
+  const size_t vec_stride = (size_t)a.Tpad;                                         // rows per head in lse2 / delta / dq_acc
+  const bool tail_kv = VARLEN && (k0 + BKV > Nk);  // rows after the tile's last valid one belong to the next sequence
 
   if (tid == 0) {
     mbar_init(bar_kv, 1);
@@ -184,6 +210,33 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     tc_fence_after();
     uint8_t* sOut = sStage + (is_dk ? 0 : SM::kKV);
     const float mul = is_dk ? a.scale : 1.f;
+    if (tail_kv) {
+      // last, partial KV tile of a packed sequence: row by row, straight from registers
+      __nv_bfloat16* dst = (is_dk ? a.dk : a.dv) + ((size_t)hk * a.total + rbase + k0 + r) * D;
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t ov[32];
+        if (N > 0 && ok) {
+          tmem_ld32(t_lane + (is_dk ? cDK : cDV) + c * 32, ov);
+          tmem_wait_ld();
+        } else {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) ov[e] = 0u;
+        }
+        if (k0 + r < Nk) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            uint4 v;
+            v.x = pack_bf16(__uint_as_float(ov[q * 8 + 0]) * mul, __uint_as_float(ov[q * 8 + 1]) * mul);
+            v.y = pack_bf16(__uint_as_float(ov[q * 8 + 2]) * mul, __uint_as_float(ov[q * 8 + 3]) * mul);
+            v.z = pack_bf16(__uint_as_float(ov[q * 8 + 4]) * mul, __uint_as_float(ov[q * 8 + 5]) * mul);
+            v.w = pack_bf16(__uint_as_float(ov[q * 8 + 6]) * mul, __uint_as_float(ov[q * 8 + 7]) * mul);
+            *reinterpret_cast<uint4*>(dst + c * 32 + q * 8) = v;
+          }
+        }
+      }
+      return;
+    }
     if (a.parts > 1) {
       // The group's heads are spread over several blocks: this block's share goes out in fp32, one slot
       // per block, and a last kernel adds the slots in a fixed order.
@@ -233,7 +286,7 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     fence_proxy_async_smem();
     wg_sync(is_dk ? 1 : 2);
     if (r == 0 && ok) {
-      for (int s = 0; s < NSLAB; ++s) tma_store_3d(is_dk ? &tmdK : &tmdV, sOut + s * SLAB_KV, s * 64, k0, bhk);
+      for (int s = 0; s < NSLAB; ++s) tma_store_3d(is_dk ? &tmdK : &tmdV, sOut + s * SLAB_KV, s * 64, rbase + k0, bhk);
       tma_commit_group();
       tma_wait_group<0>();
     }
@@ -249,8 +302,8 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         prefetch_tmap(&tmQ); prefetch_tmap(&tmdO); prefetch_tmap(&tmK); prefetch_tmap(&tmV);
         mbar_expect_tx(bar_kv, 2 * SM::kKV);
         for (int s = 0; s < NSLAB; ++s) {
-          tma_load_3d(sK + s * SLAB_KV, &tmK, bar_kv, s * 64, k0, bhk);
-          tma_load_3d(sV + s * SLAB_KV, &tmV, bar_kv, s * 64, k0, bhk);
+          tma_load_3d(sK + s * SLAB_KV, &tmK, bar_kv, s * 64, rbase + k0, bhk);
+          tma_load_3d(sV + s * SLAB_KV, &tmV, bar_kv, s * 64, rbase + k0, bhk);
         }
         int st = 0, g = 0, t_in = 0;   // stage, head of the group, position in I_h(j): kept incrementally
         uint32_t ph_e = 0;             // parity of the "stage empty" wait (the first NST steps need none)
@@ -263,11 +316,11 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           uint8_t* sdO = sQ + SM::kQS;
           mbar_expect_tx(bar_ld_full + st, SM::kStage + 512);
           for (int s = 0; s < NSLAB; ++s) {
-            tma_load_3d(sQ + s * SLAB_QS, &tmQ, bar_ld_full + st, s * 64, q0, bhq);
-            tma_load_3d(sdO + s * SLAB_QS, &tmdO, bar_ld_full + st, s * 64, q0, bhq);
+            tma_load_3d(sQ + s * SLAB_QS, &tmQ, bar_ld_full + st, s * 64, rbase + q0, bhq);
+            tma_load_3d(sdO + s * SLAB_QS, &tmdO, bar_ld_full + st, s * 64, rbase + q0, bhq);
           }
-          bulk_load_1d(sVec + st * 128, a.lse2 + (size_t)bhq * a.Tpad + q0, 256, bar_ld_full + st);
-          bulk_load_1d(sVec + st * 128 + 64, a.delta + (size_t)bhq * a.Tpad + q0, 256, bar_ld_full + st);
+          bulk_load_1d(sVec + st * 128, a.lse2 + (size_t)bhq * vec_stride + pbase + q0, 256, bar_ld_full + st);
+          bulk_load_1d(sVec + st * 128 + 64, a.delta + (size_t)bhq * vec_stride + pbase + q0, 256, bar_ld_full + st);
           if (++t_in == cnt) { t_in = 0; ++g; }
           if (++st == NST) { st = 0; if (n >= NST) ph_e ^= 1; }
         }
@@ -402,10 +455,10 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       for (int n = wg; n < N && ok; n += 2) {
         const int i = cowa_bwd_tile_at(rg, t_in);
         const int q0 = i * BQS;
-        const bool full = cowa_tile_full(w, q0, BQS, k0, BKV, off, a.Nq, a.Nk);
+        const bool full = cowa_tile_full(w, q0, BQS, k0, BKV, off, Nq, Nk);
         uint32_t mk[2] = {0xFFFFFFFFu, 0xFFFFFFFFu};
         if (!full) {
-          const long long qend = a.Nq - 1;
+          const long long qend = Nq - 1;
 #pragma unroll
           for (int c = 0; c < 2; ++c) {
             const long long base = q0 + c * 32;
@@ -413,7 +466,7 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             if (w.l > 0)
               m |= interval_bits32(kpos + w.n + w.g, min(kpos + (long long)w.n + w.g + w.l - 1, qend), base);
             if (kcol < w.s) m |= interval_bits32(kpos, qend, base);
-            mk[c] = kcol < a.Nk ? m : 0u;
+            mk[c] = kcol < Nk ? m : 0u;
           }
         }
         const float* lse2 = sVec + st * 128;
@@ -520,7 +573,7 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           fence_proxy_async_smem();
           wg_sync(3);
           if (issuer) {
-            tma_reduce_add_3d(&tmdQ, stage, 0, q0 + hf * 32, bhq);
+            tma_reduce_add_3d(&tmdQ, stage, 0, pbase + q0 + hf * 32, bhq);
             tma_commit_group();
           }
         }
@@ -590,6 +643,67 @@ __global__ void cowa_bwd_convert_dq_kernel(const float* __restrict__ acc, __nv_b
   uint4 v;
   v.x = pack_bf16(x.x, x.y); v.y = pack_bf16(x.z, x.w); v.z = pack_bf16(y.x, y.y); v.w = pack_bf16(y.z, y.w);
   *reinterpret_cast<uint4*>(dq + ((size_t)bh * T + t) * D + part * 8) = v;
+}
+
+// Packed batches.  One block per (64-row chunk of the padded row space, QO head): Delta and LSE * log2(e)
+// of the chunk's rows (padding rows: +inf, 0), read from the packed tensors.
+template <int D>
+__global__ void cowa_bwd_preprocess_varlen_kernel(const __nv_bfloat16* __restrict__ o,
+                                                  const __nv_bfloat16* __restrict__ d_o,
+                                                  const float* __restrict__ lse, float* __restrict__ lse2,
+                                                  float* __restrict__ delta, const int* __restrict__ cu, int B,
+                                                  int total, int Tpad) {
+  constexpr int TPR = D / 8;  // threads per row (16 bytes each)
+  const int chunk = blockIdx.x, h = blockIdx.y;
+  const int r = threadIdx.x / TPR, part = threadIdx.x % TPR;
+  int b, lc, nch, pb;
+  const bool in = varlen_locate(cu, B, chunk, BQS, BQS, &b, &lc, &nch, &pb);
+  const int t = lc * BQS + r;  // row inside the sequence
+  const int rbase = in ? cu[b] : 0;
+  const bool valid = in && t < cu[b + 1] - rbase && rbase >= 0 && rbase + t < total;
+  float s = 0.f;
+  if (valid) {
+    const size_t base = ((size_t)h * total + rbase + t) * D + part * 8;
+    const uint4 x = *reinterpret_cast<const uint4*>(o + base);
+    const uint4 y = *reinterpret_cast<const uint4*>(d_o + base);
+    const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      s = fmaf(__uint_as_float(xs[i] << 16), __uint_as_float(ys[i] << 16), s);
+      s = fmaf(__uint_as_float(xs[i] & 0xffff0000u), __uint_as_float(ys[i] & 0xffff0000u), s);
+    }
+  }
+#pragma unroll
+  for (int o_ = TPR / 2; o_ > 0; o_ >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o_);
+  if (part == 0) {
+    const size_t row = (size_t)h * Tpad + (size_t)chunk * BQS + r;  // chunks are laid out in order: pb == chunk * BQS
+    delta[row] = s;
+    lse2[row] = valid ? lse[(size_t)h * total + rbase + t] * 1.4426950408889634f : INFINITY;
+  }
+}
+
+// Packed batches: fp32 (or fixed-point) dQ accumulator in the padded row space -> bf16 dq in the packed one.
+template <int D>
+__global__ void cowa_bwd_convert_dq_varlen_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dq,
+                                                  const int* __restrict__ cu, int B, int total, int Tpad, int fixed) {
+  constexpr int TPR = D / 8;
+  const int chunk = blockIdx.x, h = blockIdx.y;
+  const int r = threadIdx.x / TPR, part = threadIdx.x % TPR;
+  int b, lc, nch, pb;
+  if (!varlen_locate(cu, B, chunk, BQS, BQS, &b, &lc, &nch, &pb)) return;
+  const int t = lc * BQS + r;
+  const int rbase = cu[b];
+  if (t >= cu[b + 1] - rbase || rbase < 0 || rbase + t >= total) return;
+  const float4* src = reinterpret_cast<const float4*>(acc + ((size_t)h * Tpad + (size_t)chunk * BQS + r) * D + part * 8);
+  float4 x = src[0], y = src[1];
+  if (fixed) {
+    const float u = 1.f / kDqFixedOne;
+    x = make_float4(__float_as_int(x.x) * u, __float_as_int(x.y) * u, __float_as_int(x.z) * u, __float_as_int(x.w) * u);
+    y = make_float4(__float_as_int(y.x) * u, __float_as_int(y.y) * u, __float_as_int(y.z) * u, __float_as_int(y.w) * u);
+  }
+  uint4 v;
+  v.x = pack_bf16(x.x, x.y); v.y = pack_bf16(x.z, x.w); v.z = pack_bf16(y.x, y.y); v.w = pack_bf16(y.z, y.w);
+  *reinterpret_cast<uint4*>(dq + ((size_t)h * total + rbase + t) * D + part * 8) = v;
 }
 
 // Sum of the per-block partial dK, dV (heads of a group spread over `parts` blocks), in slot order, to bf16.
@@ -709,16 +823,18 @@ int launch_bwd(const void* q, const void* k, const void* v, const void* o, const
   a.sink_tiles = 0;
   a.dq_fixed = p->deterministic ? 1 : 0;
   a.parts = parts; a.dkv_part = dkv_part;
+  a.cu = nullptr; a.dk = nullptr; a.dv = nullptr; a.total = 0; a.tiles_bound = 0;
+  a.sink = 0; a.local = 0; a.hkv_global = 0; a.hkv_offset = 0; a.full_attn = 0; a.explicit_windows = 0;
   for (int h = 0; h < Hkv; ++h) {
     const int sk = hw.w[h].s < T ? hw.w[h].s : T;
     a.sink_tiles = std::max(a.sink_tiles, (sk + BKV - 1) / BKV);
   }
-  COWA_CUDA_TRY(cudaFuncSetAttribute(cowa_bwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  COWA_CUDA_TRY(cudaFuncSetAttribute(cowa_bwd_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      BwdSmem<D>::kBytes));
   const long long nblocks = (long long)((T + BKV - 1) / BKV) * B * Hkv * parts;
   if (nblocks > 0x7FFFFFFFll) return COWA_ERR_UNSUPPORTED;
   if (g_ev_main_start) COWA_CUDA_TRY(cudaEventRecord(g_ev_main_start, st));
-  cowa_bwd_kernel<D><<<(unsigned)nblocks, 512, BwdSmem<D>::kBytes, st>>>(mq, mk, mv, mdo, mdk, mdv, mdq, a);
+  cowa_bwd_kernel<D, false><<<(unsigned)nblocks, 512, BwdSmem<D>::kBytes, st>>>(mq, mk, mv, mdo, mdk, mdv, mdq, a);
   COWA_CUDA_TRY(cudaGetLastError());
   if (g_ev_main_stop) COWA_CUDA_TRY(cudaEventRecord(g_ev_main_stop, st));
   {
@@ -737,9 +853,98 @@ int launch_bwd(const void* q, const void* k, const void* v, const void* o, const
   return COWA_OK;
 }
 
+// Padded row space of a packed batch: every sequence rounded up to 64 rows; the bound needs no lengths.
+int varlen_tpad(int B, int total) { return (total / BQS + B) * BQS; }
+
+size_t ws_bytes_varlen(int B, int total, int Hq, int D) {
+  return (size_t)Hq * varlen_tpad(B, total) * ((size_t)D + 2) * sizeof(float);
+}
+
+template <int D>
+int launch_bwd_varlen(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* d_o,
+                      void* dq, void* dk, void* dv, const int* cu, int B, int total, int Hq, int Hkv,
+                      const cowa_params_t* p, const CowaHeadWindows& hw, void* ws, cudaStream_t st) {
+  const int Tpad = varlen_tpad(B, total);
+  float* dq_acc = static_cast<float*>(ws);
+  float* lse2 = dq_acc + (size_t)Hq * Tpad * D;
+  float* delta = lse2 + (size_t)Hq * Tpad;
+  COWA_CUDA_TRY(cudaMemsetAsync(dq_acc, 0, (size_t)Hq * Tpad * D * sizeof(float), st));
+  const dim3 chunks(Tpad / BQS, Hq);
+  cowa_bwd_preprocess_varlen_kernel<D><<<chunks, BQS * (D / 8), 0, st>>>(
+      static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse, lse2, delta, cu, B, total, Tpad);
+  COWA_CUDA_TRY(cudaGetLastError());
+  CUtensorMap mq, mk, mv, mdo, mdk, mdv, mdq;
+  int rc;
+  if ((rc = cowa::make_tensor_map_3d(&mdq, dq_acc, p->deterministic ? cowa::MapType::S32 : cowa::MapType::F32, D, Tpad, Hq, D,
+                                     32, false)))
+    return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mq, q, cowa::MapType::BF16, D, total, Hq, 64, BQS))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mdo, d_o, cowa::MapType::BF16, D, total, Hq, 64, BQS))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mk, k, cowa::MapType::BF16, D, total, Hkv, 64, BKV))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mv, v, cowa::MapType::BF16, D, total, Hkv, 64, BKV))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mdk, dk, cowa::MapType::BF16, D, total, Hkv, 64, BKV))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mdv, dv, cowa::MapType::BF16, D, total, Hkv, 64, BKV))) return rc;
+  BwdArgs a;
+  a.lse2 = lse2; a.delta = delta; a.dq_acc = dq_acc;
+  a.status = cowa::device_status_word();
+  if (!a.status) return COWA_ERR_CUDA;
+  a.B = B; a.Nq = 0; a.Nk = 0; a.Hq = Hq; a.Hkv = Hkv; a.G = Hq / Hkv; a.Tpad = Tpad;
+  a.scale = p->softmax_scale;
+  a.scale_log2 = p->softmax_scale * 1.4426950408889634f;
+  a.wins = hw;
+  a.sink_tiles = 0;
+  a.dq_fixed = p->deterministic ? 1 : 0;
+  a.parts = 1; a.dkv_part = nullptr;
+  a.cu = cu; a.dk = static_cast<__nv_bfloat16*>(dk); a.dv = static_cast<__nv_bfloat16*>(dv);
+  a.total = total; a.tiles_bound = total / BKV + B;
+  a.sink = p->sink; a.local = p->local;
+  a.hkv_global = p->hkv_global > 0 ? p->hkv_global : Hkv;
+  a.hkv_offset = p->hkv_offset; a.full_attn = p->full_attn; a.explicit_windows = p->windows != nullptr;
+  COWA_CUDA_TRY(cudaFuncSetAttribute(cowa_bwd_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     BwdSmem<D>::kBytes));
+  const long long nblocks = (long long)a.tiles_bound * Hkv;
+  if (nblocks > 0x7FFFFFFFll) return COWA_ERR_UNSUPPORTED;
+  if (g_ev_main_start) COWA_CUDA_TRY(cudaEventRecord(g_ev_main_start, st));
+  cowa_bwd_kernel<D, true><<<(unsigned)nblocks, 512, BwdSmem<D>::kBytes, st>>>(mq, mk, mv, mdo, mdk, mdv, mdq, a);
+  COWA_CUDA_TRY(cudaGetLastError());
+  if (g_ev_main_stop) COWA_CUDA_TRY(cudaEventRecord(g_ev_main_stop, st));
+  cowa_bwd_convert_dq_varlen_kernel<D><<<chunks, BQS * (D / 8), 0, st>>>(dq_acc, static_cast<__nv_bfloat16*>(dq), cu, B,
+                                                                        total, Tpad, p->deterministic ? 1 : 0);
+  COWA_CUDA_TRY(cudaGetLastError());
+  return COWA_OK;
+}
+
 }  // namespace
 
 extern "C" {
+
+size_t cowa_bwd_varlen_workspace_bytes(int B, int total, int Hq, int Hkv, int D, const cowa_params_t* p) {
+  (void)p;
+  if (B <= 0 || total <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || (D != 64 && D != 128)) return 0;
+  return ws_bytes_varlen(B, total, Hq, D);
+}
+
+int cowa_bwd_varlen(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* d_o,
+                    void* dq, void* dk, void* dv, const int32_t* cu_seqlens, int B, int total, int Hq, int Hkv, int D,
+                    const cowa_params_t* p, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!q || !k || !v || !o || !lse || !d_o || !dq || !dk || !dv || !p || !workspace || !cu_seqlens)
+    return COWA_ERR_INVALID_ARG;
+  if (B <= 0 || total <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0) return COWA_ERR_INVALID_ARG;
+  if (!(p->softmax_scale > 0.f)) return COWA_ERR_INVALID_ARG;
+  if (D != 64 && D != 128) return COWA_ERR_UNSUPPORTED;
+  const void* ptrs[] = {q, k, v, o, d_o, dq, dk, dv, workspace};
+  for (const void* x : ptrs)
+    if (!cowa::aligned16(x)) return COWA_ERR_MISALIGNED;
+  if (workspace_bytes < ws_bytes_varlen(B, total, Hq, D)) return COWA_ERR_WORKSPACE_TOO_SMALL;
+  CowaHeadWindows hw;
+  int rc = cowa::resolve_windows(total, Hkv, p, &hw);  // validates; explicit tuples are copied, the default rule runs per sequence
+  if (rc != COWA_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  return D == 128 ? launch_bwd_varlen<128>(q, k, v, o, lse, d_o, dq, dk, dv, cu_seqlens, B, total, Hq, Hkv, p, hw,
+                                           workspace, st)
+                  : launch_bwd_varlen<64>(q, k, v, o, lse, d_o, dq, dk, dv, cu_seqlens, B, total, Hq, Hkv, p, hw,
+                                          workspace, st);
+}
 
 int cowa_bwd_set_profile_events(void* start_event, void* stop_event) {
   g_ev_main_start = static_cast<cudaEvent_t>(start_event);

@@ -98,32 +98,9 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   } else {
     // idx counts the QO tiles of the packed batch, sequence after sequence, each sequence's heaviest
     // (last) tile first.  Every warp finds its (sequence, tile) by a cooperative scan of the offsets.
-    const int lane = threadIdx.x & 31;
-    int base = 0;
-    b = -1; i = 0;
-    for (int b0 = 0; b0 < a.B; b0 += 32) {
-      const int bb = b0 + lane;
-      const int n = bb < a.B ? a.cu_q[bb + 1] - a.cu_q[bb] : 0;
-      const int tiles = n > 0 ? (n + BQ - 1) / BQ : 0;
-      int incl = tiles;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int y = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if (lane >= o) incl += y;
-      }
-      const int tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
-      if (idx < base + tot) {
-        const unsigned m = __ballot_sync(0xFFFFFFFFu, idx < base + incl);
-        const int src = __ffs(m) - 1;
-        const int excl = __shfl_sync(0xFFFFFFFFu, incl - tiles, src);
-        const int nt_seq = __shfl_sync(0xFFFFFFFFu, tiles, src);
-        b = b0 + src;
-        i = nt_seq - 1 - (idx - base - excl);
-        break;
-      }
-      base += tot;
-    }
-    if (b < 0) return;  // the grid is sized from an upper bound of the tile count
+    int lt, nts, pb;
+    if (!varlen_locate(a.cu_q, a.B, idx, BQ, 0, &b, &lt, &nts, &pb)) return;  // the grid is an upper bound
+    i = nts - 1 - lt;
   }
   const int h = hk * a.G + g;
   // Sequence geometry.  Packed batches: every sequence has its own N_q <= N_k, its rows start at

@@ -256,4 +256,43 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return r;
 }
 
+// Packed batches: which sequence holds tile number `idx` when every sequence b (rows cu[b] .. cu[b+1]) is
+// cut into tiles of `tile` rows, counted sequence after sequence?  Cooperative over one warp (all 32 lanes
+// must call it with the same arguments); every lane gets the same answer.  Returns false when idx is past
+// the last tile.  *pad_base is the number of rows before the sequence when every sequence is padded to a
+// multiple of `pad` rows (pad > 0).
+__device__ __forceinline__ bool varlen_locate(const int* __restrict__ cu, int B, int idx, int tile, int pad, int* b_out,
+                                              int* local_tile, int* tiles_in_seq, int* pad_base) {
+  const int lane = threadIdx.x & 31;
+  int base = 0, pbase = 0;
+  for (int b0 = 0; b0 < B; b0 += 32) {
+    const int bb = b0 + lane;
+    int n = bb < B ? cu[bb + 1] - cu[bb] : 0;
+    if (n < 0) n = 0;
+    const int tiles = (n + tile - 1) / tile;
+    const int padded = pad > 0 ? (n + pad - 1) / pad * pad : 0;
+    int incl = tiles, pincl = padded;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      const int z = __shfl_up_sync(0xFFFFFFFFu, pincl, o);
+      if (lane >= o) { incl += y; pincl += z; }
+    }
+    const int tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
+    if (idx < base + tot) {
+      const unsigned m = __ballot_sync(0xFFFFFFFFu, idx < base + incl);
+      const int src = __ffs(m) - 1;
+      const int excl = __shfl_sync(0xFFFFFFFFu, incl - tiles, src);
+      *tiles_in_seq = __shfl_sync(0xFFFFFFFFu, tiles, src);
+      *pad_base = pbase + __shfl_sync(0xFFFFFFFFu, pincl - padded, src);
+      *b_out = b0 + src;
+      *local_tile = idx - base - excl;
+      return true;
+    }
+    base += tot;
+    pbase += __shfl_sync(0xFFFFFFFFu, pincl, 31);
+  }
+  return false;
+}
+
 }  // namespace cowa_ptx

@@ -2,8 +2,10 @@
 seeded bf16 inputs.  Tolerances (bf16 inputs/outputs, fp32 accumulation, P and dS rounded to bf16
 before their second product): O and gradients max-abs 2e-2 and mean-abs 2e-3, LSE max-abs 1e-3.
 Gradients are stored as bf16 and reach magnitudes above 4, where rounding the exact value to bf16
-alone costs up to |x| * 2^-8 (half an ulp); the gradient check therefore allows
-2e-2 + 2^-8 * |reference| per element.  The mean-abs bound is unchanged."""
+alone costs up to |x| * 2^-8 (half an ulp) and |x| * 2^-10 on average (a quarter of an ulp of at
+least |x| * 2^-8); the gradient check therefore allows 2e-2 + 2^-8 * |reference| per element and
+2e-3 + 2^-10 * mean|reference| on average.  The second term only matters where most entries are
+large, e.g. a packed sequence of five tokens whose every key is attended with weight near one."""
 import numpy as np
 import pytest
 import torch
@@ -18,20 +20,21 @@ TOL_MAX, TOL_MEAN, TOL_LSE = 2e-2, 2e-3, 1e-3
 DEV = "cuda"
 
 
-def check(name, got, want, tol_max=TOL_MAX, tol_mean=TOL_MEAN, rtol=0.0):
+def check(name, got, want, tol_max=TOL_MAX, tol_mean=TOL_MEAN, rtol=0.0, rtol_mean=0.0):
     got = np.asarray(got, dtype=np.float64)
     err = np.abs(got - want)
     assert np.isfinite(got).all(), f"{name}: non-finite output"
     excess = err - rtol * np.abs(want)
     assert excess.max() <= tol_max, f"{name}: max-abs {err.max():.3e} (excess {excess.max():.3e}) > {tol_max}"
-    assert err.mean() <= tol_mean, f"{name}: mean-abs {err.mean():.3e} > {tol_mean}"
+    bound = tol_mean + rtol_mean * np.abs(want).mean()
+    assert err.mean() <= bound, f"{name}: mean-abs {err.mean():.3e} > {bound:.3e}"
 
 
 BF16_HALF_ULP = 2.0 ** -8
 
 
 def check_grad(name, got, want):
-    check(name, got, want, rtol=BF16_HALF_ULP)
+    check(name, got, want, rtol=BF16_HALF_ULP, rtol_mean=BF16_HALF_ULP / 4)
 
 
 def run_fwd(q, k, v, params):
@@ -435,6 +438,75 @@ def _full_size_sampled(name, q_tiles, kv_samples):
         dk_r, dv_r = orc.backward_dkdv_cols(qg, f(k[0, hk:hk + 1]), f(v[0, hk:hk + 1]), dog, [ws[hk]], scale, 0, cols)
         check_grad(f"{name} dk[hk{hk},tile{tile}]", dk[0, hk, cols].float().cpu().numpy(), dk_r)
         check_grad(f"{name} dv[hk{hk},tile{tile}]", dv[0, hk, cols].float().cpu().numpy(), dv_r)
+
+
+# ------------------------------------------------------------------ backward over a packed batch
+
+@pytest.mark.parametrize("lens,Hq,Hkv,D,sink,local,mode", [
+    ([100, 700, 1, 300, 128, 129, 1000], 4, 2, 128, 16, 100, "default"),
+    ([64, 65, 2048, 5], 8, 2, 64, 5, 60, "default"),
+    ([900, 333], 4, 4, 128, 8, 50, "full"),
+    ([1500, 2000, 77], 4, 2, 128, 0, 0, "explicit"),
+])
+def test_bwd_varlen(lens, Hq, Hkv, D, sink, local, mode):
+    seqs = [(n, n) for n in lens]
+    q, k, v, cu, _ = _packed_inputs(73, seqs, Hq, Hkv, D)
+    d_o = torch.cat([cowa_inputs.make_train_inputs(74 + b, 1, n, Hq, Hkv, D)[3][0] for b, n in enumerate(lens)], 1).contiguous()
+    scale = cowa_inputs.softmax_scale(D)
+    tuples = None
+    if mode == "explicit":
+        tuples = [(24, 90, 100, 400), (3, 130, 700, 900)][:Hkv]
+        params = cowa.make_params(windows=tuples, softmax_scale=scale)
+    else:
+        params = cowa.make_params(sink=sink, local=local, softmax_scale=scale, full_attn=(mode == "full"))
+    o, lse = _run_varlen(q, k, v, cu, cu, params)
+    qd, kd, vd, dod = q.to(DEV), k.to(DEV), v.to(DEV), d_o.to(DEV)
+    dq, dk, dv = (torch.full_like(x, float("nan")) for x in (qd, kd, vd))
+    total = int(cu[-1])
+    nbytes = cowa.cowa_bwd_varlen_workspace_bytes(len(lens), total, Hq, Hkv, D, params)
+    ws = torch.empty(nbytes + 64, dtype=torch.uint8, device=DEV)
+    ws.fill_(0xFF)
+    cowa.cowa_bwd_varlen(qd, kd, vd, o, lse, dod, dq, dk, dv, torch.from_numpy(cu).to(DEV), params, ws[:nbytes])
+    torch.cuda.synchronize()
+    cowa.cowa_check_device_status()
+    assert (ws[nbytes:] == 0xFF).all()
+    f = cowa_inputs.to_f64
+    for b, n in enumerate(lens):
+        if mode == "explicit":
+            wsb = tuples
+        elif mode == "full":
+            wsb = [(0, n, 0, 0)] * Hkv
+        else:
+            wsb = orc.default_windows(n, Hkv, sink, local)
+        sl = slice(cu[b], cu[b + 1])
+        dq_r, dk_r, dv_r = orc.backward(f(q[:, sl]), f(k[:, sl]), f(v[:, sl]), f(d_o[:, sl]), wsb, scale)
+        check_grad(f"varlen dq[seq {b}]", dq[:, sl].float().cpu().numpy(), dq_r)
+        check_grad(f"varlen dk[seq {b}]", dk[:, sl].float().cpu().numpy(), dk_r)
+        check_grad(f"varlen dv[seq {b}]", dv[:, sl].float().cpu().numpy(), dv_r)
+
+
+def test_bwd_varlen_equals_batched_dkdv():
+    """Equal-length sequences: dK and dV of the packed call equal the batched call's bit for bit (same block
+    arithmetic); dQ agrees within the tolerance (reduction order differs)."""
+    B, T, Hq, Hkv, D = 3, 1024, 4, 2, 128
+    q, k, v, d_o = cowa_inputs.make_train_inputs(83, B, T, Hq, Hkv, D, device=DEV)
+    params = cowa.make_params(sink=16, local=128, softmax_scale=cowa_inputs.softmax_scale(D))
+    o, lse = run_fwd(q, k, v, params)
+    dq, dk, dv = (torch.empty_like(x) for x in (q, k, v))
+    ws = torch.empty(cowa.cowa_bwd_workspace_bytes(B, T, Hq, Hkv, D, params), dtype=torch.uint8, device=DEV)
+    cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, params, ws)
+    pack = lambda x: x.permute(1, 0, 2, 3).reshape(x.shape[1], -1, x.shape[3]).contiguous()
+    cu = torch.arange(B + 1, dtype=torch.int32, device=DEV) * T
+    dq2, dk2, dv2 = (torch.empty_like(pack(x)) for x in (q, k, v))
+    ws2 = torch.empty(cowa.cowa_bwd_varlen_workspace_bytes(B, B * T, Hq, Hkv, D, params), dtype=torch.uint8, device=DEV)
+    cowa.cowa_bwd_varlen(pack(q), pack(k), pack(v), pack(o), lse.permute(1, 0, 2).reshape(Hq, -1).contiguous(), pack(d_o),
+                         dq2, dk2, dv2, cu, params, ws2)
+    torch.cuda.synchronize()
+    cowa.cowa_check_device_status()
+    if cowa.cowa_bwd_workspace_bytes(B, T, Hq, Hkv, D, params) == B * Hq * T * (D + 2) * 4:  # whole group per block
+        assert torch.equal(pack(dk), dk2) and torch.equal(pack(dv), dv2)
+    assert (pack(dk).float() - dk2.float()).abs().max().item() <= 2e-2
+    assert (pack(dq).float() - dq2.float()).abs().max().item() <= 2e-2
 
 
 def test_32k_config_sampled():
