@@ -23,6 +23,14 @@
 //                   head by head with ascending KV tile, so that the blocks in flight sweep the same
 //                   dQ rows at nearly the same time and the reductions hit in L2.
 //   3. convert      dQ accumulator (already scaled) -> bf16.
+// Two variations of the main kernel's work split:
+//   - `parts` > 1: the G heads of a group are spread over several blocks per KV tile (few tiles, or sink
+//     tiles that would be the critical path); each block writes fp32 partial dK, dV to its own slot and a
+//     fourth kernel adds the slots in order (bwd_parts, cowa_bwd_reduce_dkv_kernel).
+//   - VARLEN: packed batch [H, total, D]; a block finds (sequence, KV tile) by a warp scan of the offsets,
+//     windows follow from the sequence's own length, the accumulator and the row vectors use a row space
+//     in which every sequence is padded to 64 rows, and a sequence's last, partial KV tile is stored row
+//     by row (cowa_bwd_varlen and its own preprocess / convert kernels).
 #include <cuda_bf16.h>
 
 #include <algorithm>

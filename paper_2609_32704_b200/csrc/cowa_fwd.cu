@@ -14,6 +14,9 @@
 // result is the exact softmax.  Two blocks fit per SM (96 KB shared memory, 256 TMEM columns
 // each).  The QO heads of a GQA group at the same tile are adjacent in launch order and share
 // K/V through L2.
+// The same kernel serves N_q <= N_k (queries bottom-right aligned) and, with VARLEN, packed batches
+// [H, total, D] whose sequences have their own N_q <= N_k: a block then finds its (sequence, tile) by a
+// warp scan of the offset arrays and stores a sequence's last, partial tile row by row.
 #include <cuda_bf16.h>
 
 #include "cowa_common.h"
