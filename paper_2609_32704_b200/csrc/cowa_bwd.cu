@@ -160,10 +160,21 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     hk = idx % a.Hkv; b = idx / a.Hkv;
     w = a.wins.w[hk];
   } else {
-    // head-major: consecutive blocks are consecutive KV tiles of one head (their dQ rows overlap in L2)
-    hk = blockIdx.x / a.tiles_bound;
+    // The sink tiles of every (sequence, head) first (they meet every query tile of their sequence and are
+    // the longest blocks); then head-major: consecutive blocks are consecutive KV tiles of one head (their
+    // dQ rows overlap in L2).
+    const int nsk = a.sink_tiles, nhead = a.B * a.Hkv;
     int nts;
-    if (!varlen_locate(a.cu, a.B, blockIdx.x % a.tiles_bound, BKV, BQS, &b, &j, &nts, &pbase)) return;
+    if ((int)blockIdx.x < nsk * nhead) {
+      j = blockIdx.x / nhead;
+      b = (blockIdx.x % nhead) / a.Hkv; hk = blockIdx.x % a.Hkv;
+      varlen_seq_info(a.cu, b, BKV, BQS, &nts, &pbase);
+      if (j >= nts) return;  // the sequence is shorter than its sink
+    } else {
+      const int rest = blockIdx.x - nsk * nhead;
+      hk = rest / a.tiles_bound;
+      if (!varlen_locate(a.cu, a.B, rest % a.tiles_bound, BKV, BQS, &b, &j, &nts, &pbase, nsk)) return;
+    }
     rbase = a.cu[b];
     Nq = Nk = a.cu[b + 1] - rbase;
     if (rbase < 0 || rbase + Nk > a.total) {  // malformed offsets: report, touch nothing
@@ -900,7 +911,12 @@ int launch_bwd_varlen(const void* q, const void* k, const void* v, const void* o
   a.scale = p->softmax_scale;
   a.scale_log2 = p->softmax_scale * 1.4426950408889634f;
   a.wins = hw;
-  a.sink_tiles = 0;
+  a.sink_tiles = 0;  // KV tiles per sequence that hold sink columns (launched first)
+  if (!p->full_attn)
+    for (int h = 0; h < Hkv; ++h) {
+      const int sk = std::min(p->windows ? hw.w[h].s : p->sink, total);
+      a.sink_tiles = std::max(a.sink_tiles, (sk + BKV - 1) / BKV);
+    }
   a.dq_fixed = p->deterministic ? 1 : 0;
   a.parts = 1; a.dkv_part = nullptr;
   a.cu = cu; a.dk = static_cast<__nv_bfloat16*>(dk); a.dv = static_cast<__nv_bfloat16*>(dv);
@@ -910,7 +926,7 @@ int launch_bwd_varlen(const void* q, const void* k, const void* v, const void* o
   a.hkv_offset = p->hkv_offset; a.full_attn = p->full_attn; a.explicit_windows = p->windows != nullptr;
   COWA_CUDA_TRY(cudaFuncSetAttribute(cowa_bwd_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      BwdSmem<D>::kBytes));
-  const long long nblocks = (long long)a.tiles_bound * Hkv;
+  const long long nblocks = (long long)a.tiles_bound * Hkv + (long long)a.sink_tiles * B * Hkv;
   if (nblocks > 0x7FFFFFFFll) return COWA_ERR_UNSUPPORTED;
   if (g_ev_main_start) COWA_CUDA_TRY(cudaEventRecord(g_ev_main_start, st));
   cowa_bwd_kernel<D, true><<<(unsigned)nblocks, 512, BwdSmem<D>::kBytes, st>>>(mq, mk, mv, mdo, mdk, mdv, mdq, a);

@@ -260,16 +260,17 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // cut into tiles of `tile` rows, counted sequence after sequence?  Cooperative over one warp (all 32 lanes
 // must call it with the same arguments); every lane gets the same answer.  Returns false when idx is past
 // the last tile.  *pad_base is the number of rows before the sequence when every sequence is padded to a
-// multiple of `pad` rows (pad > 0).
+// multiple of `pad` rows (pad > 0).  With skip > 0 the first `skip` tiles of every sequence are left out of
+// the count (they are handed out separately); *local_tile still counts from the sequence's first tile.
 __device__ __forceinline__ bool varlen_locate(const int* __restrict__ cu, int B, int idx, int tile, int pad, int* b_out,
-                                              int* local_tile, int* tiles_in_seq, int* pad_base) {
+                                              int* local_tile, int* tiles_in_seq, int* pad_base, int skip = 0) {
   const int lane = threadIdx.x & 31;
   int base = 0, pbase = 0;
   for (int b0 = 0; b0 < B; b0 += 32) {
     const int bb = b0 + lane;
     int n = bb < B ? cu[bb + 1] - cu[bb] : 0;
     if (n < 0) n = 0;
-    const int tiles = (n + tile - 1) / tile;
+    const int tiles = max((n + tile - 1) / tile - skip, 0);
     const int padded = pad > 0 ? (n + pad - 1) / pad * pad : 0;
     int incl = tiles, pincl = padded;
 #pragma unroll
@@ -283,16 +284,35 @@ __device__ __forceinline__ bool varlen_locate(const int* __restrict__ cu, int B,
       const unsigned m = __ballot_sync(0xFFFFFFFFu, idx < base + incl);
       const int src = __ffs(m) - 1;
       const int excl = __shfl_sync(0xFFFFFFFFu, incl - tiles, src);
-      *tiles_in_seq = __shfl_sync(0xFFFFFFFFu, tiles, src);
+      *tiles_in_seq = __shfl_sync(0xFFFFFFFFu, tiles, src) + skip;
       *pad_base = pbase + __shfl_sync(0xFFFFFFFFu, pincl - padded, src);
       *b_out = b0 + src;
-      *local_tile = idx - base - excl;
+      *local_tile = skip + idx - base - excl;
       return true;
     }
     base += tot;
     pbase += __shfl_sync(0xFFFFFFFFu, pincl, 31);
   }
   return false;
+}
+
+// Companion of varlen_locate for a known sequence b: its tile count and its padded row base (warp-cooperative).
+__device__ __forceinline__ void varlen_seq_info(const int* __restrict__ cu, int b, int tile, int pad, int* tiles_in_seq,
+                                                int* pad_base) {
+  const int lane = threadIdx.x & 31;
+  int sum = 0;
+  for (int b0 = 0; b0 < b; b0 += 32) {
+    const int bb = b0 + lane;
+    int n = bb < b ? cu[bb + 1] - cu[bb] : 0;
+    if (n < 0) n = 0;
+    sum += (n + pad - 1) / pad * pad;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+  int n = cu[b + 1] - cu[b];
+  if (n < 0) n = 0;
+  *tiles_in_seq = (n + tile - 1) / tile;
+  *pad_base = sum;
 }
 
 }  // namespace cowa_ptx
