@@ -64,7 +64,7 @@ struct DecodeArgs {
   const int32_t* block_table;  // [B, max_pages] page of every page_size-row stretch of a sequence, or nullptr
   int NQ;                      // query tokens per sequence, at key positions lens[b] - NQ .. lens[b] - 1
   int tpg, ngroups;            // tokens per block (columns = tpg * Hq / Hkv <= 8), blocks per (sequence, KV head)
-  int page_size, max_pages;
+  int page_size, max_pages, page_shift;  // page_shift = log2(page_size) when that is a power of two, else -1
 };
 
 // Position of the v-th visible row (v in the concatenation of the head's ranges).
@@ -134,8 +134,11 @@ __global__ void __launch_bounds__(kThreads, 5) cowa_decode_split_kernel(const De
   auto row_ptr = [&](const __nv_bfloat16* base, int tok) -> const __nv_bfloat16* {
     if constexpr (EXT) {
       if (a.block_table) {
-        const int pg = a.block_table[(size_t)b * a.max_pages + tok / a.page_size];
-        return base + (((size_t)pg * a.Hkv + hk) * a.page_size + tok % a.page_size) * D;
+        // page sizes are almost always powers of two: shift and mask instead of a runtime division
+        const int pi = a.page_shift >= 0 ? tok >> a.page_shift : tok / a.page_size;
+        const int po = a.page_shift >= 0 ? tok & (a.page_size - 1) : tok % a.page_size;
+        const int pg = a.block_table[(size_t)b * a.max_pages + pi];
+        return base + (((size_t)pg * a.Hkv + hk) * a.page_size + po) * D;
       }
     }
     return base + ((size_t)b * a.Hkv + hk) * (size_t)a.Tmax * D + (size_t)tok * D;
@@ -529,7 +532,7 @@ int decode_launch(const void* q, const void* kc, const void* vc, const int32_t* 
   a.hkv_offset = p->hkv_offset;
   a.full_attn = p->full_attn;
   a.scale_log2 = p->softmax_scale * 1.4426950408889634f;
-  a.block_table = nullptr; a.NQ = 1; a.tpg = 1; a.ngroups = 1; a.page_size = 0; a.max_pages = 0;
+  a.block_table = nullptr; a.NQ = 1; a.tpg = 1; a.ngroups = 1; a.page_size = 0; a.max_pages = 0; a.page_shift = -1;
   const int G = Hq / Hkv;
   cudaError_t e = (D == 128) ? dispatch_split<128, false>(G, a, st) : dispatch_split<64, false>(G, a, st);
   if (e != cudaSuccess) return record_cuda_error(e);
@@ -560,6 +563,10 @@ int decode_ext_launch(const void* q, const void* kc, const void* vc, const int32
   a.full_attn = p->full_attn;
   a.scale_log2 = p->softmax_scale * 1.4426950408889634f;
   a.block_table = block_table; a.NQ = NQ; a.page_size = page_size; a.max_pages = max_pages;
+  a.page_shift = -1;
+  if (page_size > 0 && (page_size & (page_size - 1)) == 0)
+    for (int sft = 0; sft < 31; ++sft)
+      if ((1 << sft) == page_size) a.page_shift = sft;
   int cols;
   token_groups(NQ, Hq / Hkv, &a.tpg, &a.ngroups, &cols);
   cudaError_t e = (D == 128) ? dispatch_split<128, true>(cols, a, st) : dispatch_split<64, true>(cols, a, st);

@@ -710,6 +710,7 @@ def test_decode_multi_full_attn():
     (2, 4, 4100, 8, 4, 128, 32, 200, [4100, 999], 64),
     (2, 2, 8192, 16, 2, 64, 128, 512, [8192, 640], 256),
     (1, 1, 40000, 4, 2, 128, 128, 4096, [39999], 128),
+    (2, 3, 3000, 4, 2, 128, 16, 100, [3000, 1111], 48),    # page size not a power of two
 ])
 def test_decode_paged_shapes(B, Nq, Tmax, Hq, Hkv, D, sink, local, lens, page):
     multi_case(B, Nq, Tmax, Hq, Hkv, D, sink, local, lens, page_size=page)
