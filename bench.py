@@ -610,7 +610,15 @@ def run_cuda(args):
         "bwd_ms": bwd_ms if have_bwd else None, "bwd_tflops": bwd_flops / bwd_ms / 1e9 if have_bwd else None,
         "bwd_main_kernel_ms": bwd_main_ms,
         "visited_tiles": cnt["visited"], "causal_tiles": cnt["causal"],
-        "decode": decode, "prefill_varlen": varlen, "decode_variants": dec_var, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
+        "decode": decode, "prefill_varlen": varlen, "decode_variants": dec_var, "roofline": roofline,
+        "roofline_other_kernels": [
+            {"kernel": "cowa_fwd_kernel<128, 0>", "bound": "tensor", "achieved": fwd_flops / fwd_ms / 1e9, "peak": peak_tf,
+             "unit": "TFLOP/s", "frac": fwd_flops / fwd_ms / 1e9 / peak_tf,
+             "frac_of_burst_peak": fwd_flops / fwd_ms / 1e9 / peaks["bf16_tflops"],
+             "traffic": traffic_128k.get("cowa_fwd_kernel<128, 0>") if args.train_cfg == "128k" else None},
+            {"kernel": "cowa_decode_split_kernel<128, 4, 0> + merge", "bound": "hbm", "achieved": b2b_gbs,
+             "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": b2b_gbs / peaks["hbm_gbs"],
+             "traffic": 0.615e9 if not args.decode_batch else None}], "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
         "gpu_launches": args.steps * (1 + (BWD_LAUNCHES if have_bwd else 0) + 2),
     }
     line.update(full)
