@@ -188,7 +188,8 @@ size_t cowa_decode_static_capacity(void);
  *   kcache, vcache [B,Hkv,Tmax,D] already hold the Nq new tokens; lens: DEVICE int32[B], Nq <= lens[b] <= Tmax.
  * 1 <= Nq <= 64; Hq/Hkv in {1,2,4,8}.  Tokens are packed into the 8 columns of the score MMA together with
  * the group's heads: 8/(Hq/Hkv) tokens share one pass over the visible rows, more tokens take more blocks
- * (their re-reads mostly hit in L2).  `workspace`: device, >= cowa_decode_multi_workspace_bytes, 16-byte
+ * (their re-reads mostly hit in L2; beyond about three such passes cowa_prefill / cowa_prefill_varlen, whose
+ * cost does not grow with Nq up to 128, is the faster call).  `workspace`: device, >= cowa_decode_multi_workspace_bytes, 16-byte
  * aligned, no initialisation needed.  cowa_params_t.windows is ignored, as in cowa_decode. */
 int cowa_decode_multi(const void* q, const void* kcache, const void* vcache, const int32_t* lens,
                       void* o, float* lse, int B, int Nq, int Tmax, int Hq, int Hkv, int D,
