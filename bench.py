@@ -588,7 +588,7 @@ def run_cuda(args):
                                "calls": n_dec}}
 
     cpu = None
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and world == 1:  # the oracle is timed on one-GPU runs only
         f, t, units = oracle_sample(args.cpu_seconds)
         cpu = {"value": f / t / 1e12, "unit": "TFLOP/s", "cores": cpu_threads(), "kind": "oracle",
                "sample": f"oracle forward of {units} random (KV head, 128-row query tile) units of the 128K "
