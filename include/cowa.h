@@ -232,8 +232,9 @@ int cowa_equal_area_windows(int Nq, int Nk, int Hkv_global, int hkv_offset, int 
  * kernels' scheduler computes, as an int32 stream into the HOST buffer `out`:
  *   COWA_SCHED_FWD    for each head h, QO tile i:  h, i, n, then n pairs (j, full) with j descending
  *   COWA_SCHED_BWD    for each head h, KV tile j:  h, j, n, then n pairs (i, full) with i ascending
- *   COWA_SCHED_DECODE (Nq must be 1) for each head h: h, r, then r pairs (start, end) of visible key
- *                     ranges [start,end) ascending, then m, then m visited block_k-block indices
+ *   COWA_SCHED_DECODE for each head h: h, r, then r pairs (start, end) of visible key ranges [start,end)
+ *                     ascending, then m, then m visited block_k-block indices; Nq = 1 is the decode step,
+ *                     Nq > 1 the union over the Nq newest tokens (what cowa_decode_multi streams)
  * full = 1 when every pair of the nominal block_q x block_k tile is legal, else 0 (boundary tile).
  * *out_len receives the number of int32 needed; COWA_ERR_WORKSPACE_TOO_SMALL if out_cap is less
  * (nothing beyond out_cap is written). */

@@ -104,7 +104,6 @@ int cowa_schedule_dump(int which, int Nq, int Nk, int Hkv, const cowa_params_t* 
                        size_t out_cap, size_t* out_len) {
   if (!p || !out_len || Nq <= 0 || Nk <= 0 || Nq > Nk || Hkv <= 0) return COWA_ERR_INVALID_ARG;
   if (p->block_q <= 0 || p->block_k <= 0) return COWA_ERR_INVALID_ARG;
-  if (which == COWA_SCHED_DECODE && Nq != 1) return COWA_ERR_INVALID_ARG;
   if (Hkv > COWA_MAX_HKV) return COWA_ERR_UNSUPPORTED;
   CowaHeadWindows hw;
   int st = cowa::resolve_windows(Nk, Hkv, p, &hw);
@@ -146,7 +145,7 @@ int cowa_schedule_dump(int which, int Nq, int Nk, int Hkv, const cowa_params_t* 
       }
     } else if (which == COWA_SCHED_DECODE) {
       CowaRange r[3];
-      const int nr = cowa_decode_ranges(w, Nk, r);
+      const int nr = Nq == 1 ? cowa_decode_ranges(w, Nk, r) : cowa_decode_ranges_span(w, Nk - Nq, Nk - 1, r);
       put(h); put(nr);
       for (int t = 0; t < nr; ++t) { put(r[t].lo); put(r[t].hi + 1); }
       // visited blocks: the blocks touched by the ranges, each once

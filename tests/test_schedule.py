@@ -191,6 +191,24 @@ def test_decode_schedule():
             assert got[hk] == (ranges, blocks), (Nk, hk)
 
 
+def test_decode_schedule_of_several_newest_tokens():
+    """Union of the keys the Nq newest tokens see (what the multi-token decode kernel streams), from the
+    oracle's explicit mask of those Nq query rows."""
+    for Nk, Nq, Hkv, sink, near, Bk in [(5000, 2, 4, 16, 100, 64), (777, 5, 4, 5, 60, 64), (4230, 8, 8, 128, 4096, 128),
+                                        (300, 3, 2, 0, 7, 16), (64, 64, 2, 3, 9, 16), (1000, 4, 8, 40, 40, 32)]:
+        p = cowa.make_params(sink=sink, local=near, block=Bk)
+        got = parse_decode(cowa.cowa_schedule_dump(cowa.SCHED_DECODE, Nq, Nk, Hkv, p))
+        for hk, w in enumerate(orc.default_windows(Nk, Hkv, sink, near)):
+            seen = orc.visible_mask(Nq, Nk, w).any(axis=0)
+            idx = np.flatnonzero(seen)
+            cuts = np.flatnonzero(np.diff(idx) > 1)
+            starts = np.concatenate([[idx[0]], idx[cuts + 1]])
+            ends = np.concatenate([idx[cuts], [idx[-1]]]) + 1
+            ranges = [(int(a_), int(b_)) for a_, b_ in zip(starts, ends)]
+            blocks = sorted(set(int(i) // Bk for i in idx))
+            assert got[hk] == (ranges, blocks), (Nk, Nq, hk)
+
+
 def test_argument_validation_without_gpu():
     L = cowa.lib()
     p = cowa.make_params(sink=1, local=0)
