@@ -242,11 +242,43 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     float m_ref = -INFINITY, l_sum = 0.f;
     const float2 sc2 = make_float2(a.scale_log2, a.scale_log2);
 
+    // Which visited tiles need no mask?  Inside each of the three ranges these form one interval of tile
+    // indices, found once here; the loop then only compares.  The intervals are conservative (a tile that
+    // straddles two windows, or sink and non-sink columns, is treated as a boundary tile and masked, which
+    // is always correct).  With d = (row position) - (key index): every pair of tile j is causal iff
+    // 64 j + 63 <= q0 + off; it lies in the near window iff q1 + off - 64 j < n; in the long window iff also
+    // q0 + off - (64 j + 63) >= n + g and q1 + off - 64 j < n + g + l; in the sink iff 64 j + 63 < s.
+    int f_lo[3] = {1, 1, 1}, f_hi[3] = {0, 0, 0};
+    if (q0 + BQ <= Nq) {
+      auto fdiv = [](long long x) -> int { return (int)(x >= 0 ? x / BK : -((-x + BK - 1) / BK)); };
+      const long long p0 = (long long)q0 + off, p1 = p0 + BQ - 1;
+      const int causal_hi = fdiv(p0 - (BK - 1));
+      f_lo[0] = fdiv(p1 - w.n) + 1; f_hi[0] = causal_hi;
+      if (w.l > 0) {
+        f_lo[1] = fdiv(p1 - ((long long)w.n + w.g + w.l)) + 1;
+        f_hi[1] = min(causal_hi, fdiv(p0 - ((long long)w.n + w.g) - (BK - 1)));
+      }
+      f_lo[2] = 0; f_hi[2] = min(causal_hi, w.s >= BK ? (w.s - BK) / BK : -1);
+    }
+    // walk of the ranges: tile j steps down to j_last, then the next non-empty range is entered; the
+    // current range's bounds live in registers (selects, no indexed local arrays)
+    int rr = -1, j = 0, j_last = 0, fl = 1, fh = 0;
+    auto next_range = [&]() {
+#pragma unroll
+      for (int c = 0; c < 3; ++c) {
+        if (rr < c && rg[c].hi >= rg[c].lo) {
+          rr = c; j = rg[c].hi; j_last = rg[c].lo; fl = f_lo[c]; fh = f_hi[c];
+          return;
+        }
+      }
+      rr = 3;
+    };
+    next_range();
+
     for (int t = 0; t < nt && ok; ++t) {
       const int b_ = t & 1;
-      const int j = cowa_fwd_tile_at(rg, t);
       const int k0 = j * BK;
-      const bool full = cowa_tile_full(w, q0, BQ, k0, BK, off, Nq, Nk);
+      const bool full = j >= fl && j <= fh;
       const uint32_t t_S = t_lane + b_ * 64;
 
       ok = mbar_wait(bar_s + b_, (t >> 1) & 1, a.status);
@@ -328,6 +360,7 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(bar_p + b_);
+      if (j > j_last) --j; else next_range();
     }
 
     // ---- epilogue: O / l, LSE ----
