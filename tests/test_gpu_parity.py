@@ -731,3 +731,82 @@ def test_decode_multi_last_token_equals_single_token_decode():
     o1, lse1 = run_decode(q[:, Nq - 1].contiguous(), kc, vc, lens, params)
     assert (o[:, Nq - 1].float() - o1.float()).abs().max().item() <= 1e-2
     assert (lse[:, Nq - 1] - lse1).abs().max().item() <= 1e-4
+
+
+# ------------------------------------------------------------------ seeded random shapes
+
+def _random_tuples(rng, T, Hkv):
+    """Explicit per-head tuples with arbitrary sinks, gaps and widths (possibly overlapping, possibly beyond T)."""
+    return [(int(rng.integers(0, 200)), int(rng.integers(1, 300)), int(rng.integers(0, T)), int(rng.integers(0, T)))
+            for _ in range(Hkv)]
+
+
+@pytest.mark.parametrize("case", range(24))
+def test_random_shapes(case):
+    """Forward, backward and decode on shapes drawn from a fixed seed: odd lengths, every supported group size,
+    default rule and arbitrary explicit tuples."""
+    rng = np.random.default_rng(1000 + case)
+    D = int(rng.choice([64, 128]))
+    Hkv = int(rng.choice([1, 2, 3, 4]))
+    G = int(rng.choice([1, 2, 4, 8]))
+    Hq = Hkv * G
+    B = int(rng.integers(1, 3))
+    T = int(rng.integers(1, 1400))
+    sink, local = int(rng.integers(0, 150)), int(rng.integers(1, 400))
+    windows = _random_tuples(rng, T, Hkv) if case % 3 == 2 else None
+    fwd_case(B, T, Hq, Hkv, D, sink, local, seed=300 + case, windows=windows)
+    bwd_case(B, T, Hq, Hkv, D, sink, local, seed=300 + case, windows=windows)
+    lens = [int(rng.integers(1, T + 1)) for _ in range(B)]
+    decode_case(B, T, Hq, Hkv, D, sink, local, lens, seed=400 + case)
+    nq = int(rng.integers(1, 6))
+    multi_case(B, nq, T + nq, Hq, Hkv, D, sink, local, [n + nq - 1 for n in lens], seed=500 + case,
+               page_size=(16 * int(rng.integers(1, 9)) if case % 2 else None))
+
+
+@pytest.mark.parametrize("case", range(6))
+def test_random_packed_batches(case):
+    """Packed forward (N_q <= N_k per sequence) and packed backward (N_q = N_k) on random length mixes."""
+    rng = np.random.default_rng(2000 + case)
+    D = int(rng.choice([64, 128]))
+    Hkv = int(rng.choice([1, 2, 4]))
+    Hq = Hkv * int(rng.choice([1, 2, 4]))
+    sink, local = int(rng.integers(0, 100)), int(rng.integers(1, 300))
+    nseq = int(rng.integers(1, 7))
+    seqs = []
+    for _ in range(nseq):
+        nk = int(rng.integers(1, 900))
+        seqs.append((int(rng.integers(0, nk + 1)), nk))
+    if all(nq == 0 for nq, _ in seqs):
+        seqs[0] = (seqs[0][1], seqs[0][1])
+    scale = cowa_inputs.softmax_scale(D)
+    params = cowa.make_params(sink=sink, local=local, softmax_scale=scale)
+    q, k, v, cu_q, cu_k = _packed_inputs(600 + 20 * case, seqs, Hq, Hkv, D)
+    o, lse = _run_varlen(q, k, v, cu_q, cu_k, params)
+    cowa.cowa_check_device_status()
+    f = cowa_inputs.to_f64
+    for b, (nq, nk) in enumerate(seqs):
+        if nq == 0:
+            continue
+        qs, ks = slice(cu_q[b], cu_q[b + 1]), slice(cu_k[b], cu_k[b + 1])
+        o_ref, lse_ref = orc.forward(f(q[:, qs]), f(k[:, ks]), f(v[:, ks]), orc.default_windows(nk, Hkv, sink, local), scale)
+        check(f"packed lse[seq {b}]", lse[:, qs].cpu().numpy(), lse_ref, TOL_LSE, TOL_LSE)
+        check(f"packed o[seq {b}]", o[:, qs].float().cpu().numpy(), o_ref)
+    # backward on the same key lengths with N_q = N_k
+    lens = [nk for _, nk in seqs]
+    q, k, v, cu, _ = _packed_inputs(700 + 20 * case, [(n, n) for n in lens], Hq, Hkv, D)
+    d_o = torch.cat([cowa_inputs.make_train_inputs(800 + b, 1, n, Hq, Hkv, D)[3][0] for b, n in enumerate(lens)], 1).contiguous()
+    o, lse = _run_varlen(q, k, v, cu, cu, params)
+    qd, kd, vd, dod = q.to(DEV), k.to(DEV), v.to(DEV), d_o.to(DEV)
+    dq, dk, dv = (torch.full_like(x, float("nan")) for x in (qd, kd, vd))
+    ws = torch.empty(cowa.cowa_bwd_varlen_workspace_bytes(len(lens), int(cu[-1]), Hq, Hkv, D, params), dtype=torch.uint8,
+                     device=DEV)
+    cowa.cowa_bwd_varlen(qd, kd, vd, o, lse, dod, dq, dk, dv, torch.from_numpy(cu).to(DEV), params, ws)
+    torch.cuda.synchronize()
+    cowa.cowa_check_device_status()
+    for b, n in enumerate(lens):
+        sl = slice(cu[b], cu[b + 1])
+        dq_r, dk_r, dv_r = orc.backward(f(q[:, sl]), f(k[:, sl]), f(v[:, sl]), f(d_o[:, sl]),
+                                        orc.default_windows(n, Hkv, sink, local), scale)
+        check_grad(f"packed dq[seq {b}]", dq[:, sl].float().cpu().numpy(), dq_r)
+        check_grad(f"packed dk[seq {b}]", dk[:, sl].float().cpu().numpy(), dk_r)
+        check_grad(f"packed dv[seq {b}]", dv[:, sl].float().cpu().numpy(), dv_r)
