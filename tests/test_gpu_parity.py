@@ -810,3 +810,51 @@ def test_random_packed_batches(case):
         check_grad(f"packed dq[seq {b}]", dq[:, sl].float().cpu().numpy(), dq_r)
         check_grad(f"packed dk[seq {b}]", dk[:, sl].float().cpu().numpy(), dk_r)
         check_grad(f"packed dv[seq {b}]", dv[:, sl].float().cpu().numpy(), dv_r)
+
+
+# ------------------------------------------------------------------ CUDA graphs
+
+def test_calls_replay_from_a_cuda_graph():
+    """The library's launches (kernels, the accumulator memset, the programmatic dependent launch of the decode
+    merge) can be captured into a CUDA graph after one warm-up call, and the replay reproduces the direct
+    call bit for bit on new inputs written into the same buffers."""
+    B, T, Hq, Hkv, D = 2, 1536, 8, 2, 128
+    params = cowa.make_params(sink=16, local=128, softmax_scale=cowa_inputs.softmax_scale(D), deterministic=True)
+    q, k, v, d_o = cowa_inputs.make_train_inputs(91, B, T, Hq, Hkv, D, device=DEV)
+    o = torch.empty_like(q)
+    lse = torch.empty((B, Hq, T), dtype=torch.float32, device=DEV)
+    dq, dk, dv = (torch.empty_like(x) for x in (q, k, v))
+    ws = torch.empty(cowa.cowa_bwd_workspace_bytes(B, T, Hq, Hkv, D, params), dtype=torch.uint8, device=DEV)
+    qd = q[:, :, -1].contiguous()
+    od = torch.empty_like(qd)
+    lsed = torch.empty((B, Hq), dtype=torch.float32, device=DEV)
+    lens = torch.tensor([T, T - 300], dtype=torch.int32, device=DEV)
+    wsd = torch.empty(cowa.cowa_decode_workspace_bytes(B, T, Hq, Hkv, D, params), dtype=torch.uint8, device=DEV)
+
+    def step():
+        cowa.cowa_fwd(q, k, v, o, lse, params)
+        cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, params, ws)
+        cowa.cowa_decode(qd, k, v, lens, od, lsed, params, wsd)
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        step()                                   # warm-up outside the capture
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            step()
+    torch.cuda.synchronize()
+    # new inputs in place, then direct call vs replay
+    q2, k2, v2, d_o2 = cowa_inputs.make_train_inputs(92, B, T, Hq, Hkv, D, device=DEV)
+    q.copy_(q2); k.copy_(k2); v.copy_(v2); d_o.copy_(d_o2); qd.copy_(q2[:, :, -1])
+    step()
+    torch.cuda.synchronize()
+    want = [x.clone() for x in (o, lse, dq, dk, dv, od, lsed)]
+    for x in (o, lse, dq, dk, dv, od, lsed):
+        x.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    cowa.cowa_check_device_status()
+    for name, a_, b_ in zip(("o", "lse", "dq", "dk", "dv", "o_decode", "lse_decode"), (o, lse, dq, dk, dv, od, lsed), want):
+        assert torch.equal(a_, b_), name
