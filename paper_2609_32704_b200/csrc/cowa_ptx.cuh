@@ -1,5 +1,5 @@
 // Thin inline-PTX wrappers for the sm_100a features the training kernels use: mbarrier,
-// TMA tiled copies (no multicast anywhere), tcgen05 MMA / TMEM access, shared-memory and
+// TMA tiled copies (each block loads its own tiles), tcgen05 MMA / TMEM access, shared-memory and
 // instruction descriptors.  Device-only.
 #pragma once
 #include <cuda.h>
