@@ -125,6 +125,16 @@ int cowa_bwd(const void* q, const void* k, const void* v, const void* o, const f
  * on the call's stream (both are cudaEvent_t handles owned by the caller; NULL, NULL switches it off). */
 int cowa_bwd_set_profile_events(void* start_event, void* stop_event);
 
+/* Backward of cowa_prefill: the same Algorithm 2 with N_q <= N_k (queries bottom-right aligned, Eq.
+ * fwa_distance; windows from N_k).  q, o, d_o, dq [B,Hq,Nq,D]; k, v, dk, dv [B,Hkv,Nk,D]; lse [B,Hq,Nq].
+ * Keys no query sees get zero gradients.  cowa_bwd is this call with Nq = Nk = T; workspace size from
+ * cowa_bwd_prefill_workspace_bytes. */
+int cowa_bwd_prefill(const void* q, const void* k, const void* v, const void* o, const float* lse,
+                     const void* d_o, void* dq, void* dk, void* dv,
+                     int B, int Nq, int Nk, int Hq, int Hkv, int D, const cowa_params_t* p,
+                     void* workspace, size_t workspace_bytes, void* stream);
+size_t cowa_bwd_prefill_workspace_bytes(int B, int Nq, int Nk, int Hq, int Hkv, int D, const cowa_params_t* p);
+
 /* Training backward over a packed batch of B sequences of different lengths (self-attention: N_q = N_k =
  * the sequence's length; Algorithm 2 applied per sequence, each with windows from its own length, Sec. 2.1).
  *   q, o, d_o, dq [Hq,total,D]; k, v, dk, dv [Hkv,total,D] bf16; lse [Hq,total] fp32 as written by

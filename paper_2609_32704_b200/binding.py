@@ -54,6 +54,10 @@ def lib():
         L.cowa_prefill_varlen.restype = i32
         L.cowa_bwd.argtypes = [vp] * 9 + [i32] * 5 + [pp, vp, sz, vp]
         L.cowa_bwd.restype = i32
+        L.cowa_bwd_prefill.argtypes = [vp] * 9 + [i32] * 6 + [pp, vp, sz, vp]
+        L.cowa_bwd_prefill.restype = i32
+        L.cowa_bwd_prefill_workspace_bytes.argtypes = [i32] * 6 + [pp]
+        L.cowa_bwd_prefill_workspace_bytes.restype = sz
         L.cowa_bwd_varlen.argtypes = [vp] * 10 + [i32] * 5 + [pp, vp, sz, vp]
         L.cowa_bwd_varlen.restype = i32
         L.cowa_bwd_varlen_workspace_bytes.argtypes = [i32] * 5 + [pp]
@@ -190,6 +194,23 @@ def cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, params, workspace):
     _check(lib().cowa_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(d_o), _ptr(dq), _ptr(dk),
                           _ptr(dv), B, T, Hq, Hkv, D, C.byref(params), _ptr(workspace),
                           workspace.numel() * workspace.element_size(), _stream()), "cowa_bwd")
+
+
+def cowa_bwd_prefill_workspace_bytes(B, Nq, Nk, Hq, Hkv, D, params):
+    return int(lib().cowa_bwd_prefill_workspace_bytes(B, Nq, Nk, Hq, Hkv, D, C.byref(params)))
+
+
+def cowa_bwd_prefill(q, k, v, o, lse, d_o, dq, dk, dv, params, workspace):
+    """Backward with N_q <= N_k: q/o/d_o/dq [B,Hq,Nq,D], k/v/dk/dv [B,Hkv,Nk,D], lse [B,Hq,Nq]."""
+    import torch
+    for t, n in ((q, "q"), (k, "k"), (v, "v"), (o, "o"), (d_o, "d_o"), (dq, "dq"), (dk, "dk"), (dv, "dv")):
+        _need(t, torch.bfloat16, n)
+    _need(lse, torch.float32, "lse")
+    B, Hq, Nq, D = q.shape
+    Hkv, Nk = k.shape[1], k.shape[2]
+    _check(lib().cowa_bwd_prefill(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(d_o), _ptr(dq), _ptr(dk),
+                                  _ptr(dv), B, Nq, Nk, Hq, Hkv, D, C.byref(params), _ptr(workspace),
+                                  workspace.numel() * workspace.element_size(), _stream()), "cowa_bwd_prefill")
 
 
 def cowa_bwd_varlen_workspace_bytes(B, total, Hq, Hkv, D, params):

@@ -771,14 +771,14 @@ thread_local cudaEvent_t g_ev_main_start = nullptr, g_ev_main_stop = nullptr;
 // are spread over `parts` blocks (a divisor of G), chosen as the smallest that gives two waves of
 // blocks and keeps the longest block under 3/4 of an even share of the work.
 constexpr int kSMs = 148;
-int bwd_parts(int B, int T, int Hkv, int G, const CowaHeadWindows& hw) {
-  const int nKV = (T + BKV - 1) / BKV;
+int bwd_parts(int B, int Nq, int Nk, int Hkv, int G, const CowaHeadWindows& hw) {
+  const int nKV = (Nk + BKV - 1) / BKV;
   long long total = 0, longest = 0;
   for (int h = 0; h < Hkv; ++h)
     for (int j = 0; j < nKV; ++j) {
       CowaRange rg[2];
-      const int k0 = j * BKV, k1 = std::min(k0 + BKV, T) - 1;
-      cowa_bwd_ranges(hw.w[h], k0, k1, 0, T, BQS, rg);
+      const int k0 = j * BKV, k1 = std::min(k0 + BKV, Nk) - 1;
+      cowa_bwd_ranges(hw.w[h], k0, k1, Nk - Nq, Nq, BQS, rg);
       const long long cnt = cowa_range_len(rg[0]) + cowa_range_len(rg[1]);
       total += cnt;
       longest = std::max(longest, cnt);
@@ -793,20 +793,21 @@ int bwd_parts(int B, int T, int Hkv, int G, const CowaHeadWindows& hw) {
   return G;
 }
 
-size_t part_bytes(int B, int T, int Hkv, int D, int parts) {
+size_t part_bytes(int B, int Nk, int Hkv, int D, int parts) {
   if (parts <= 1) return 0;
-  return (size_t)B * Hkv * ((T + BKV - 1) / BKV) * parts * 2 * BKV * D * sizeof(float);
+  return (size_t)B * Hkv * ((Nk + BKV - 1) / BKV) * parts * 2 * BKV * D * sizeof(float);
 }
 
-size_t ws_bytes(int B, int T, int Hq, int Hkv, int D, int parts) {
-  const size_t Tpad = ((size_t)T + BQS - 1) / BQS * BQS;
-  return (size_t)B * Hq * Tpad * ((size_t)D + 2) * sizeof(float) + part_bytes(B, T, Hkv, D, parts);
+size_t ws_bytes(int B, int Nq, int Nk, int Hq, int Hkv, int D, int parts) {
+  const size_t Tpad = ((size_t)Nq + BQS - 1) / BQS * BQS;
+  return (size_t)B * Hq * Tpad * ((size_t)D + 2) * sizeof(float) + part_bytes(B, Nk, Hkv, D, parts);
 }
 
 template <int D>
 int launch_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* d_o,
-               void* dq, void* dk, void* dv, int B, int T, int Hq, int Hkv, const cowa_params_t* p,
+               void* dq, void* dk, void* dv, int B, int Nq, int Nk, int Hq, int Hkv, const cowa_params_t* p,
                const CowaHeadWindows& hw, int parts, void* ws, cudaStream_t st) {
+  const int T = Nq;  // rows of q, o, d_o, dq, lse
   const int Tpad = (T + BQS - 1) / BQS * BQS;
   const long long BH = (long long)B * Hq;
   float* dq_acc = static_cast<float*>(ws);
@@ -827,15 +828,15 @@ int launch_bwd(const void* q, const void* k, const void* v, const void* o, const
     return rc;
   if ((rc = cowa::make_tensor_map_3d(&mq, q, cowa::MapType::BF16, D, T, BH, 64, BQS))) return rc;
   if ((rc = cowa::make_tensor_map_3d(&mdo, d_o, cowa::MapType::BF16, D, T, BH, 64, BQS))) return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mk, k, cowa::MapType::BF16, D, T, (long long)B * Hkv, 64, BKV))) return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mv, v, cowa::MapType::BF16, D, T, (long long)B * Hkv, 64, BKV))) return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mdk, dk, cowa::MapType::BF16, D, T, (long long)B * Hkv, 64, BKV))) return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mdv, dv, cowa::MapType::BF16, D, T, (long long)B * Hkv, 64, BKV))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mk, k, cowa::MapType::BF16, D, Nk, (long long)B * Hkv, 64, BKV))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mv, v, cowa::MapType::BF16, D, Nk, (long long)B * Hkv, 64, BKV))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mdk, dk, cowa::MapType::BF16, D, Nk, (long long)B * Hkv, 64, BKV))) return rc;
+  if ((rc = cowa::make_tensor_map_3d(&mdv, dv, cowa::MapType::BF16, D, Nk, (long long)B * Hkv, 64, BKV))) return rc;
   BwdArgs a;
   a.lse2 = lse2; a.delta = delta; a.dq_acc = dq_acc;
   a.status = cowa::device_status_word();
   if (!a.status) return COWA_ERR_CUDA;
-  a.B = B; a.Nq = T; a.Nk = T; a.Hq = Hq; a.Hkv = Hkv; a.G = Hq / Hkv; a.Tpad = Tpad;
+  a.B = B; a.Nq = Nq; a.Nk = Nk; a.Hq = Hq; a.Hkv = Hkv; a.G = Hq / Hkv; a.Tpad = Tpad;
   a.scale = p->softmax_scale;
   a.scale_log2 = p->softmax_scale * 1.4426950408889634f;
   a.wins = hw;
@@ -845,12 +846,12 @@ int launch_bwd(const void* q, const void* k, const void* v, const void* o, const
   a.cu = nullptr; a.dk = nullptr; a.dv = nullptr; a.total = 0; a.tiles_bound = 0;
   a.sink = 0; a.local = 0; a.hkv_global = 0; a.hkv_offset = 0; a.full_attn = 0; a.explicit_windows = 0;
   for (int h = 0; h < Hkv; ++h) {
-    const int sk = hw.w[h].s < T ? hw.w[h].s : T;
+    const int sk = hw.w[h].s < Nk ? hw.w[h].s : Nk;
     a.sink_tiles = std::max(a.sink_tiles, (sk + BKV - 1) / BKV);
   }
   COWA_CUDA_TRY(cudaFuncSetAttribute(cowa_bwd_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      BwdSmem<D>::kBytes));
-  const long long nblocks = (long long)((T + BKV - 1) / BKV) * B * Hkv * parts;
+  const long long nblocks = (long long)((Nk + BKV - 1) / BKV) * B * Hkv * parts;
   if (nblocks > 0x7FFFFFFFll) return COWA_ERR_UNSUPPORTED;
   if (g_ev_main_start) COWA_CUDA_TRY(cudaEventRecord(g_ev_main_start, st));
   cowa_bwd_kernel<D, false><<<(unsigned)nblocks, 512, BwdSmem<D>::kBytes, st>>>(mq, mk, mv, mdo, mdk, mdv, mdq, a);
@@ -863,10 +864,10 @@ int launch_bwd(const void* q, const void* k, const void* v, const void* o, const
     COWA_CUDA_TRY(cudaGetLastError());
   }
   if (parts > 1) {
-    const int nKV = (T + BKV - 1) / BKV;
+    const int nKV = (Nk + BKV - 1) / BKV;
     const long long threads = (long long)B * Hkv * nKV * BKV * (D / 8);
     cowa_bwd_reduce_dkv_kernel<D><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(
-        dkv_part, static_cast<__nv_bfloat16*>(dk), static_cast<__nv_bfloat16*>(dv), T, nKV, parts, (long long)B * Hkv);
+        dkv_part, static_cast<__nv_bfloat16*>(dk), static_cast<__nv_bfloat16*>(dv), Nk, nKV, parts, (long long)B * Hkv);
     COWA_CUDA_TRY(cudaGetLastError());
   }
   return COWA_OK;
@@ -976,31 +977,41 @@ int cowa_bwd_set_profile_events(void* start_event, void* stop_event) {
   return COWA_OK;
 }
 
-size_t cowa_bwd_workspace_bytes(int B, int T, int Hq, int Hkv, int D, const cowa_params_t* p) {
-  if (B <= 0 || T <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || D <= 0 || !p) return 0;
+size_t cowa_bwd_prefill_workspace_bytes(int B, int Nq, int Nk, int Hq, int Hkv, int D, const cowa_params_t* p) {
+  if (B <= 0 || Nq <= 0 || Nk < Nq || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || D <= 0 || !p) return 0;
   CowaHeadWindows hw;
-  if (cowa::resolve_windows(T, Hkv, p, &hw) != COWA_OK) return 0;
-  return ws_bytes(B, T, Hq, Hkv, D, bwd_parts(B, T, Hkv, Hq / Hkv, hw));
+  if (cowa::resolve_windows(Nk, Hkv, p, &hw) != COWA_OK) return 0;
+  return ws_bytes(B, Nq, Nk, Hq, Hkv, D, bwd_parts(B, Nq, Nk, Hkv, Hq / Hkv, hw));
 }
 
-int cowa_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* d_o,
-             void* dq, void* dk, void* dv, int B, int T, int Hq, int Hkv, int D, const cowa_params_t* p,
-             void* workspace, size_t workspace_bytes, void* stream) {
+size_t cowa_bwd_workspace_bytes(int B, int T, int Hq, int Hkv, int D, const cowa_params_t* p) {
+  return cowa_bwd_prefill_workspace_bytes(B, T, T, Hq, Hkv, D, p);
+}
+
+int cowa_bwd_prefill(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* d_o,
+                     void* dq, void* dk, void* dv, int B, int Nq, int Nk, int Hq, int Hkv, int D,
+                     const cowa_params_t* p, void* workspace, size_t workspace_bytes, void* stream) {
   if (!q || !k || !v || !o || !lse || !d_o || !dq || !dk || !dv || !p || !workspace) return COWA_ERR_INVALID_ARG;
-  if (B <= 0 || T <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0) return COWA_ERR_INVALID_ARG;
+  if (B <= 0 || Nq <= 0 || Nk < Nq || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0) return COWA_ERR_INVALID_ARG;
   if (!(p->softmax_scale > 0.f)) return COWA_ERR_INVALID_ARG;
   if (D != 64 && D != 128) return COWA_ERR_UNSUPPORTED;
   const void* ptrs[] = {q, k, v, o, d_o, dq, dk, dv, workspace};
   for (const void* x : ptrs)
     if (!cowa::aligned16(x)) return COWA_ERR_MISALIGNED;
   CowaHeadWindows hw;
-  int rc = cowa::resolve_windows(T, Hkv, p, &hw);
+  int rc = cowa::resolve_windows(Nk, Hkv, p, &hw);
   if (rc != COWA_OK) return rc;
-  const int parts = bwd_parts(B, T, Hkv, Hq / Hkv, hw);
-  if (workspace_bytes < ws_bytes(B, T, Hq, Hkv, D, parts)) return COWA_ERR_WORKSPACE_TOO_SMALL;
+  const int parts = bwd_parts(B, Nq, Nk, Hkv, Hq / Hkv, hw);
+  if (workspace_bytes < ws_bytes(B, Nq, Nk, Hq, Hkv, D, parts)) return COWA_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  return D == 128 ? launch_bwd<128>(q, k, v, o, lse, d_o, dq, dk, dv, B, T, Hq, Hkv, p, hw, parts, workspace, st)
-                  : launch_bwd<64>(q, k, v, o, lse, d_o, dq, dk, dv, B, T, Hq, Hkv, p, hw, parts, workspace, st);
+  return D == 128 ? launch_bwd<128>(q, k, v, o, lse, d_o, dq, dk, dv, B, Nq, Nk, Hq, Hkv, p, hw, parts, workspace, st)
+                  : launch_bwd<64>(q, k, v, o, lse, d_o, dq, dk, dv, B, Nq, Nk, Hq, Hkv, p, hw, parts, workspace, st);
+}
+
+int cowa_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* d_o,
+             void* dq, void* dk, void* dv, int B, int T, int Hq, int Hkv, int D, const cowa_params_t* p,
+             void* workspace, size_t workspace_bytes, void* stream) {
+  return cowa_bwd_prefill(q, k, v, o, lse, d_o, dq, dk, dv, B, T, T, Hq, Hkv, D, p, workspace, workspace_bytes, stream);
 }
 
 }  // extern "C"

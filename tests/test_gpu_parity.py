@@ -440,6 +440,41 @@ def _full_size_sampled(name, q_tiles, kv_samples):
         check_grad(f"{name} dv[hk{hk},tile{tile}]", dv[0, hk, cols].float().cpu().numpy(), dv_r)
 
 
+# ------------------------------------------------------------------ backward with N_q < N_k
+
+@pytest.mark.parametrize("B,Nq,Nk,Hq,Hkv,D,sink,local", [
+    (1, 256, 1024, 4, 2, 128, 16, 100),    # a chunk appended to an existing cache
+    (2, 100, 777, 8, 2, 64, 5, 60),        # ragged sizes
+    (1, 1, 900, 4, 2, 128, 32, 200),       # one query
+    (1, 513, 514, 2, 1, 128, 0, 7),        # off = 1, H_k = 1
+    (1, 300, 3000, 8, 4, 128, 64, 256),    # far bands clipped; most keys seen by no query of their head
+])
+def test_bwd_prefill_shapes(B, Nq, Nk, Hq, Hkv, D, sink, local):
+    q, _, _, d_o = cowa_inputs.make_train_inputs(55, B, Nq, Hq, Hkv, D)
+    _, k, v, _ = cowa_inputs.make_train_inputs(56, B, Nk, Hq, Hkv, D)
+    scale = cowa_inputs.softmax_scale(D)
+    params = cowa.make_params(sink=sink, local=local, softmax_scale=scale)
+    qd, kd, vd, dod = q.to(DEV), k.to(DEV), v.to(DEV), d_o.to(DEV)
+    o = torch.empty_like(qd)
+    lse = torch.empty((B, Hq, Nq), dtype=torch.float32, device=DEV)
+    cowa.cowa_prefill(qd, kd, vd, o, lse, params)
+    dq, dk, dv = (torch.full_like(x, float("nan")) for x in (qd, kd, vd))
+    nbytes = cowa.cowa_bwd_prefill_workspace_bytes(B, Nq, Nk, Hq, Hkv, D, params)
+    ws = torch.empty(nbytes + 64, dtype=torch.uint8, device=DEV)
+    ws.fill_(0xFF)
+    cowa.cowa_bwd_prefill(qd, kd, vd, o, lse, dod, dq, dk, dv, params, ws[:nbytes])
+    torch.cuda.synchronize()
+    cowa.cowa_check_device_status()
+    assert (ws[nbytes:] == 0xFF).all()
+    wins = orc.default_windows(Nk, Hkv, sink, local)
+    f = cowa_inputs.to_f64
+    for b in range(B):
+        dq_r, dk_r, dv_r = orc.backward(f(q[b]), f(k[b]), f(v[b]), f(d_o[b]), wins, scale)
+        check_grad(f"prefill dq[b={b}]", dq[b].float().cpu().numpy(), dq_r)
+        check_grad(f"prefill dk[b={b}]", dk[b].float().cpu().numpy(), dk_r)
+        check_grad(f"prefill dv[b={b}]", dv[b].float().cpu().numpy(), dv_r)
+
+
 # ------------------------------------------------------------------ backward over a packed batch
 
 @pytest.mark.parametrize("lens,Hq,Hkv,D,sink,local,mode", [
