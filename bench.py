@@ -41,6 +41,35 @@ def load_peaks():
     return dict(FALLBACK_PEAKS), "fallback"
 
 
+def load_traffic():
+    """DRAM bytes per launch of the kernels, from the tracked ncu summary file profiles/traffic.json:
+    {kernel name: {"bytes_per_launch": ..., "workload": ..., "source": ...}}.  Missing file or kernel: None."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    if not os.path.exists(path):
+        return {}
+    with open(path) as f:
+        return json.load(f)
+
+
+def traffic_for(table, kernel, workload):
+    e = table.get(kernel)
+    if not e or e.get("workload") != workload:
+        return None
+    return e.get("bytes_per_launch")
+
+
+def tp_shards(rank, world, tp):
+    """KV-head shards of a TP group of `tp` ranks that process `rank` of `world` times: its own shard when
+    world == tp, every world-th shard when fewer processes than shards run, none for surplus processes."""
+    return list(range(rank, tp, world))
+
+
+def duplicated_windows(windows, m):
+    """Control layout of the collective-coverage study: head h gets the band of head h mod m of the default
+    layout (every head keeps the shared sink and near windows)."""
+    return [windows[h % m] for h in range(len(windows))]
+
+
 class ClockSampler:
     """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
 
@@ -241,7 +270,11 @@ def run_cuda(args):
         cd["B"] = args.decode_batch
     B, T, Hq, Hkv, D = ct["B"], ct["T"], ct["Hq"], ct["Hkv"], ct["D"]
     scale = cowa_inputs.softmax_scale(D)
-    p_train = cowa.make_params(sink=ct["sink"], local=ct["local"], softmax_scale=scale,
+    train_windows = None
+    if args.windows != "default":  # duplicated-window control: the first m bands repeated over the heads
+        m = int(args.windows[3:])
+        train_windows = duplicated_windows(cowa.cowa_default_windows(T, Hkv, 0, Hkv, ct["sink"], ct["local"]), m)
+    p_train = cowa.make_params(sink=ct["sink"], local=ct["local"], softmax_scale=scale, windows=train_windows,
                                deterministic=args.deterministic)
     p_full = cowa.make_params(softmax_scale=scale, full_attn=True, deterministic=args.deterministic)
     p_dec = cowa.make_params(sink=cd["sink"], local=cd["local"], softmax_scale=scale)
@@ -264,7 +297,7 @@ def run_cuda(args):
     cnt = cowa.cowa_tile_counts(T, T, Hkv, p_train)
     cnt_full = cowa.cowa_tile_counts(T, T, Hkv, p_full)
     G = Hq // Hkv
-    legal_pairs = count_legal_pairs(T, cowa.cowa_default_windows(T, Hkv, 0, Hkv, ct["sink"], ct["local"]))
+    legal_pairs = count_legal_pairs(T, train_windows or cowa.cowa_default_windows(T, Hkv, 0, Hkv, ct["sink"], ct["local"]))
     fwd_flops = cnt["visited"] * 128 * 128 * 4 * D * G * B
     bwd_flops = 2.5 * fwd_flops
     full_fwd_flops = cnt_full["visited"] * 128 * 128 * 4 * D * G * B
@@ -275,13 +308,8 @@ def run_cuda(args):
             vis_rows += min(n, w_[0] + w_[1] + w_[3])
     dec_bytes = vis_rows * cd["D"] * 2 * 2
 
-    have_bwd = True
-    try:
-        cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, p_train, ws_bwd)
-    except cowa.CowaError as e:
-        if e.status != -2:
-            raise
-        have_bwd = False
+    have_bwd = True  # every phase is part of the step; a failing call raises
+    cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, p_train, ws_bwd)
     torch.cuda.synchronize()
 
     main_evs = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
@@ -294,9 +322,8 @@ def run_cuda(args):
         cowa.cowa_fwd(q, k, v, o, lse, params)
         if ev: ev[1].record()
         if have_bwd:
-            if main_ev: cowa.cowa_bwd_set_profile_events(main_ev[0], main_ev[1])
-            cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, params, ws_bwd)
-            if main_ev: cowa.cowa_bwd_set_profile_events(None, None)
+            pb = cowa.with_bwd_events(params, main_ev[0], main_ev[1]) if main_ev else params
+            cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, pb, ws_bwd)
         if ev: ev[2].record()
         cowa.cowa_decode(qd, kc, vc, lens, od, lsed, p_dec, ws_dec)
         if ev: ev[3].record()
@@ -389,38 +416,57 @@ def run_cuda(args):
         cowa.cowa_check_device_status()
         del kp, vp
 
-    # ---- FullAttn path of the same library (few iterations: it is ~5.4x the work) ----
+    # ---- FullAttn path of the same library: the same step (forward, backward, decode in that order), one
+    # warm-up step and three timed ones (it is ~5.4x the work), so that every ratio compares like with like ----
     full = {}
     if rank == 0 and not args.no_fullattn:
-        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
-        cowa.cowa_fwd(q, k, v, o, lse, p_full)
-        torch.cuda.synchronize()
-        e[0].record()
-        cowa.cowa_fwd(q, k, v, o, lse, p_full)
-        e[1].record()
-        if have_bwd:
-            cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, p_full, ws_bwd)
-        e[2].record()
-        torch.cuda.synchronize()
-        f_ms, b_ms = e[0].elapsed_time(e[1]), e[1].elapsed_time(e[2])
-        full = {"fullattn_fwd_ms": f_ms, "fullattn_fwd_tflops": full_fwd_flops / f_ms / 1e9,
-                "speedup_fwd": f_ms / fwd_ms, "work_ratio_tiles": cnt_full["visited"] / cnt["visited"]}
-        if have_bwd:
-            full.update({"fullattn_bwd_ms": b_ms, "speedup_bwd": b_ms / bwd_ms})
-        # decode FullAttn: every head reads the whole prefix
         ws_df = torch.empty(cowa.cowa_decode_workspace_bytes(cd["B"], cd["Tmax"], cd["Hq"], cd["Hkv"], cd["D"], p_full),
                             dtype=torch.uint8, device=dev)
-        cowa.cowa_decode(qd, kc, vc, lens, od, lsed, p_full, ws_df)
+        n_full = 3
+
+        def full_step(ev=None):
+            if ev: ev[0].record()
+            cowa.cowa_fwd(q, k, v, o, lse, p_full)
+            if ev: ev[1].record()
+            cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, p_full, ws_bwd)
+            if ev: ev[2].record()
+            cowa.cowa_decode(qd, kc, vc, lens, od, lsed, p_full, ws_df)
+            if ev: ev[3].record()
+
+        full_step()
         torch.cuda.synchronize()
+        fe = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(n_full)]
+        for e_ in fe:
+            full_step(e_)
+        torch.cuda.synchronize()
+        f_ms = sum(e_[0].elapsed_time(e_[1]) for e_ in fe) / n_full
+        b_ms = sum(e_[1].elapsed_time(e_[2]) for e_ in fe) / n_full
+        fd_step_ms = sum(e_[2].elapsed_time(e_[3]) for e_ in fe) / n_full
         e2 = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        for _ in range(2):
+            cowa.cowa_decode(qd, kc, vc, lens, od, lsed, p_full, ws_df)
         e2[0].record()
         for _ in range(5):
             cowa.cowa_decode(qd, kc, vc, lens, od, lsed, p_full, ws_df)
         e2[1].record()
         torch.cuda.synchronize()
-        fd_ms = e2[0].elapsed_time(e2[1]) / 5
-        full.update({"fullattn_decode_us": fd_ms * 1e3, "speedup_decode": fd_ms / dec_ms,
-                     "byte_ratio_decode": sum(lens_h) * cd["Hkv"] / vis_rows})
+        fd_b2b_ms = e2[0].elapsed_time(e2[1]) / 5
+        tile_ratio = cnt_full["visited"] / cnt["visited"]
+        byte_ratio = sum(lens_h) * cd["Hkv"] / vis_rows
+        # the bar of the speed-up criterion: CoWA time <= FullAttn time x (visited / causal work) x 1.2
+        full = {"fullattn_iterations": n_full,
+                "fullattn_fwd_ms": f_ms, "fullattn_fwd_tflops": full_fwd_flops / f_ms / 1e9,
+                "fullattn_bwd_ms": b_ms, "fullattn_bwd_tflops": 2.5 * full_fwd_flops / b_ms / 1e9,
+                "speedup_fwd": f_ms / fwd_ms, "speedup_bwd": b_ms / bwd_ms, "work_ratio_tiles": tile_ratio,
+                "bar_fwd_ms": 1.2 * f_ms / tile_ratio, "bar_bwd_ms": 1.2 * b_ms / tile_ratio,
+                "meets_bar_fwd": fwd_ms <= 1.2 * f_ms / tile_ratio, "meets_bar_bwd": bwd_ms <= 1.2 * b_ms / tile_ratio,
+                "fullattn_decode_us_in_step": fd_step_ms * 1e3, "fullattn_decode_us_back_to_back": fd_b2b_ms * 1e3,
+                "speedup_decode_in_step": fd_step_ms / dec_ms, "speedup_decode_back_to_back": fd_b2b_ms / dec_b2b_ms,
+                "byte_ratio_decode": byte_ratio,
+                "bar_decode_us_in_step": 1.2e3 * fd_step_ms / byte_ratio,
+                "bar_decode_us_back_to_back": 1.2e3 * fd_b2b_ms / byte_ratio,
+                "meets_bar_decode_in_step": dec_ms <= 1.2 * fd_step_ms / byte_ratio,
+                "meets_bar_decode_back_to_back": dec_b2b_ms <= 1.2 * fd_b2b_ms / byte_ratio}
         del ws_df
 
     # ---- prefill over a packed batch of mixed lengths (one launch) against one call per sequence ----
@@ -489,6 +535,15 @@ def run_cuda(args):
             varlen.update({"bwd_ms": b_ms, "bwd_tflops": 2.5 * v_flops / b_ms / 1e9})
             del pdo, pdq, pdk, pdv, wsv
         del pq, pk, pv, po, plse
+
+    # ---- the other training configurations beside FullAttn, and the slowest TP=8 shard at 128K ----
+    table, tp_row = None, None
+    if rank == 0 and not args.no_table:
+        table = [train_config_row(cowa, cowa_inputs, name, mode, dev)
+                 for name, mode in (("tiny", "default"), ("8k", "default"), ("8k", "dup1"), ("32k", "default"))]
+        tp_row = tp_replica_rows(cowa, cowa_inputs, dev, [131072], 0, 1, 3, 3)[0]
+        tp_row["note"] = ("TP=8 shards of the paper's benchmark shape (Hq=64, Hkv=8, D=128, sink+near=128+896), timed "
+                          "one after another on this GPU; slowest shard per phase")
 
     # ---- end to end: host buffers in, results back to the host, copies inside the timed region ----
     e2e = None
@@ -564,20 +619,22 @@ def run_cuda(args):
         return
 
     # ---- roofline of the dominant kernel ----
-    if have_bwd and bwd_ms >= fwd_ms:
-        dom, dom_flops, dom_ms = "cowa_bwd_kernel<128>", bwd_flops, bwd_main_ms
+    k_fwd, k_bwd, k_dec = f"cowa_fwd_kernel<{D}, 0>", f"cowa_bwd_kernel<{D}, 0>", f"cowa_decode_split_kernel<{cd['D']}, {cd['Hq'] // cd['Hkv']}, 0>"
+    if bwd_ms >= fwd_ms:
+        dom, dom_flops, dom_ms = k_bwd, bwd_flops, bwd_main_ms
     else:
-        dom, dom_flops, dom_ms = "cowa_fwd_kernel<128, 0>", fwd_flops, fwd_ms
+        dom, dom_flops, dom_ms = k_fwd, fwd_flops, fwd_ms
     peak_tf = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
     achieved = dom_flops / dom_ms / 1e9
-    # DRAM bytes per launch of the dominant kernel at the 128K workload: dram__bytes_read.sum +
-    # dram__bytes_write.sum of a one-pass ncu capture of this same command.
-    traffic_128k = {"cowa_bwd_kernel<128>": 12.904e9 + 6.795e9, "cowa_fwd_kernel<128, 0>": 9.546e9 + 1.055e9}
+    # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum of an ncu capture) come from the
+    # tracked summary profiles/traffic.json, keyed by kernel name and workload; no entry, no number.
+    traffic = load_traffic()
+    wl = args.train_cfg if args.windows == "default" else None
     roofline = {"kernel": dom, "bound": "tensor", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s",
                 "frac": achieved / peak_tf, "peak_source": f"{peak_src} bf16 sustained (kernel timed inside a long step)",
                 "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "frac_of_nominal_2250": achieved / 2250.0,
-                "traffic": traffic_128k.get(dom) if args.train_cfg == "128k" else None,
-                "traffic_unit": "bytes per launch (ncu, 128K workload)"}
+                "traffic": traffic_for(traffic, dom, wl),
+                "traffic_unit": "bytes per launch (ncu; see profiles/traffic.json for the capture it comes from)"}
     dec_gbs = dec_bytes / (dec_ms * 1e-3) / 1e9
     b2b_gbs = dec_bytes / (dec_b2b_ms * 1e-3) / 1e9
     decode = {"us_per_step": dec_ms * 1e3, "us_per_token": dec_ms * 1e3 / cd["B"], "visible_kv_bytes": dec_bytes,
@@ -599,7 +656,7 @@ def run_cuda(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": args.train_cfg, "decode_workload": DECODE_CFG, "decode_batch": cd["B"], "B": B, "T": T, "Hq": Hq, "Hkv": Hkv,
-                   "D": D, "sink": ct["sink"], "near": ct["local"], "deterministic_dq": bool(args.deterministic),
+                   "D": D, "sink": ct["sink"], "near": ct["local"], "deterministic_dq": bool(args.deterministic), "windows": args.windows,
                    "phases": ["fwd"] + (["bwd"] if have_bwd else []) + ["decode"],
                    "l2": "inputs larger than L2 (2.6 GB training tensors, 0.57 GB visible KV cache)",
                    "parallelism": "independent replicas" if world > 1 else "single GPU"},
@@ -612,13 +669,15 @@ def run_cuda(args):
         "visited_tiles": cnt["visited"], "causal_tiles": cnt["causal"],
         "decode": decode, "prefill_varlen": varlen, "decode_variants": dec_var, "roofline": roofline,
         "roofline_other_kernels": [
-            {"kernel": "cowa_fwd_kernel<128, 0>", "bound": "tensor", "achieved": fwd_flops / fwd_ms / 1e9, "peak": peak_tf,
+            {"kernel": k_fwd, "bound": "tensor", "achieved": fwd_flops / fwd_ms / 1e9, "peak": peak_tf,
              "unit": "TFLOP/s", "frac": fwd_flops / fwd_ms / 1e9 / peak_tf,
              "frac_of_burst_peak": fwd_flops / fwd_ms / 1e9 / peaks["bf16_tflops"],
-             "traffic": traffic_128k.get("cowa_fwd_kernel<128, 0>") if args.train_cfg == "128k" else None},
-            {"kernel": "cowa_decode_split_kernel<128, 4, 0> + merge", "bound": "hbm", "achieved": b2b_gbs,
+             "traffic": traffic_for(traffic, k_fwd, wl)},
+            {"kernel": k_dec + " + merge", "bound": "hbm", "achieved": b2b_gbs,
              "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": b2b_gbs / peaks["hbm_gbs"],
-             "traffic": 0.615e9 if not args.decode_batch else None}], "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
+             "frac_nominal_8tbs": b2b_gbs / 8000.0,
+             "traffic": traffic_for(traffic, k_dec, DECODE_CFG if not args.decode_batch else None)}],
+        "configs_table": table, "tp_replica": tp_row, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
         "gpu_launches": args.steps * (1 + (BWD_LAUNCHES if have_bwd else 0) + 2),
     }
     line.update(full)
@@ -639,6 +698,103 @@ PAPER_TP8_MS = {
 }
 
 
+def timed_ms(torch, fn, warmup, iters, flush=None):
+    for _ in range(warmup):
+        fn()
+    tot = 0.0
+    for _ in range(iters):
+        if flush is not None:
+            flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); fn(); e1.record()
+        torch.cuda.synchronize()
+        tot += e0.elapsed_time(e1)
+    return tot / iters
+
+
+def train_config_row(cowa, cowa_inputs, name, mode, dev, warmup=2, iters=5):
+    """Forward and backward of one training configuration, CoWA (or the duplicated-window control) beside
+    FullAttn at the same shape: ms, speed-up, and the visited / causal tile ratio the speed-up is held against."""
+    import torch
+    c = cowa_inputs.CONFIGS[name]
+    B, T, Hq, Hkv, D = c["B"], c["T"], c["Hq"], c["Hkv"], c["D"]
+    scale = cowa_inputs.softmax_scale(D)
+    wins = None
+    if mode != "default":
+        wins = duplicated_windows(cowa.cowa_default_windows(T, Hkv, 0, Hkv, c["sink"], c["local"]), int(mode[3:]))
+    p = cowa.make_params(sink=c["sink"], local=c["local"], softmax_scale=scale, windows=wins)
+    pf = cowa.make_params(softmax_scale=scale, full_attn=True)
+    q, k, v, d_o = cowa_inputs.make_train_inputs(c["index"], B, T, Hq, Hkv, D, device=dev)
+    o = torch.empty_like(q)
+    lse = torch.empty((B, Hq, T), dtype=torch.float32, device=dev)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    ws = torch.empty(max(cowa.cowa_bwd_workspace_bytes(B, T, Hq, Hkv, D, p), cowa.cowa_bwd_workspace_bytes(B, T, Hq, Hkv, D, pf), 16),
+                     dtype=torch.uint8, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if q.numel() * 2 < (128 << 20) else None
+    row = {"config": name, "windows": mode, "B": B, "T": T, "Hq": Hq, "Hkv": Hkv, "D": D,
+           "l2": "flushed before every timed call" if flush is not None else "inputs larger than L2"}
+    cnt, cntf = cowa.cowa_tile_counts(T, T, Hkv, p), cowa.cowa_tile_counts(T, T, Hkv, pf)
+    flops = cnt["visited"] * 128 * 128 * 4 * D * (Hq // Hkv) * B
+    for tag, par in (("cowa", p), ("fullattn", pf)):
+        row[tag + "_fwd_ms"] = timed_ms(torch, lambda: cowa.cowa_fwd(q, k, v, o, lse, par), warmup, iters, flush)
+        row[tag + "_bwd_ms"] = timed_ms(torch, lambda: cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, par, ws), warmup, iters, flush)
+    cowa.cowa_check_device_status()
+    row.update({"fwd_tflops": flops / row["cowa_fwd_ms"] / 1e9, "bwd_tflops": 2.5 * flops / row["cowa_bwd_ms"] / 1e9,
+                "speedup_fwd": row["fullattn_fwd_ms"] / row["cowa_fwd_ms"],
+                "speedup_bwd": row["fullattn_bwd_ms"] / row["cowa_bwd_ms"],
+                "tile_ratio": cntf["visited"] / cnt["visited"], "visited_tiles": cnt["visited"], "causal_tiles": cnt["causal"],
+                "iterations": iters})
+    return row
+
+
+def tp_replica_rows(cowa, cowa_inputs, dev, lengths, rank, world, warmup, iters):
+    """Per sequence length: the slowest TP=8 shard per phase and layout among the shards this process owns."""
+    import torch
+    TP, Hq_r, D, sink, near = 8, 8, 128, 128, 896
+    scale = cowa_inputs.softmax_scale(D)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    rows = []
+    for T in lengths:
+        q, k, v, d_o = cowa_inputs.make_train_inputs(11, 1, T, Hq_r, 1, D, device=dev)
+        o = torch.empty_like(q)
+        lse = torch.empty((1, Hq_r, T), dtype=torch.float32, device=dev)
+        dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+        qd, od = q[:, :, -1].contiguous(), torch.empty((1, Hq_r, D), dtype=torch.bfloat16, device=dev)
+        lsed = torch.empty((1, Hq_r), dtype=torch.float32, device=dev)
+        lens = torch.tensor([T], dtype=torch.int32, device=dev)
+        worst = {}
+        for layout in ("cowa", "eq", "full"):  # default equal-width bands, equal-area bands, dense
+            for r in tp_shards(rank, world, TP):
+                if layout == "eq":
+                    p = cowa.make_params(windows=cowa.cowa_equal_area_windows(T, T, TP, r, 1, sink, near),
+                                         softmax_scale=scale)
+                else:
+                    p = cowa.make_params(sink=sink, local=near, softmax_scale=scale, full_attn=(layout == "full"),
+                                         hkv_global=TP, hkv_offset=r)
+                ws = torch.empty(max(cowa.cowa_bwd_workspace_bytes(1, T, Hq_r, 1, D, p), 16), dtype=torch.uint8,
+                                 device=dev)
+                wsd = torch.empty(max(cowa.cowa_decode_workspace_bytes(1, T, Hq_r, 1, D, p), 16), dtype=torch.uint8,
+                                  device=dev)
+                t = {"fwd": timed_ms(torch, lambda: cowa.cowa_fwd(q, k, v, o, lse, p), warmup, iters, flush),
+                     "bwd": timed_ms(torch, lambda: cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, p, ws), warmup, iters, flush)}
+                if layout != "eq":  # decode keeps the equal-width rule (Sec. 2.1), so there is no third variant
+                    t["dec"] = timed_ms(torch, lambda: cowa.cowa_decode(qd, k, v, lens, od, lsed, p, wsd), warmup, iters, flush)
+                for ph, ms in t.items():
+                    key = layout + "_" + ph
+                    worst[key] = max(worst.get(key, 0.0), ms)
+                if layout == "full":
+                    break  # dense shards are identical on every rank
+        cowa.cowa_check_device_status()
+        rows.append({"T": T, **{k_ + "_ms": v_ for k_, v_ in sorted(worst.items())}})
+        del q, k, v, d_o, o, lse, dq, dk, dv
+    return rows
+
+
+def reduce_worst(rows, world):
+    """Slowest shard over all ranks, per phase (every rank passes the rows of its own shards)."""
+    return [{k_: (max_over_ranks(v_, world) if k_.endswith("_ms") else v_) for k_, v_ in sorted(r.items())} for r in rows]
+
+
 def run_tp_replica(args):
     """Each rank of a TP=8 group owns one KV head and its 8 QO heads and runs the operator on its
     shard without any exchange; the group's latency is the slowest rank's.  With fewer than 8 GPUs
@@ -652,76 +808,26 @@ def run_tp_replica(args):
         raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
     rank, world, _ = dist_setup(args.gpus)
     dev = torch.device("cuda", torch.cuda.current_device())
-    TP, Hq_r, D, sink, near = 8, 8, 128, 128, 896
-    scale = cowa_inputs.softmax_scale(D)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-    iters = max(args.steps, 3)
-
-    def timed(fn):
-        for _ in range(max(args.warmup, 3)):
-            fn()
-        tot = 0.0
-        for _ in range(iters):
-            flush.fill_(1)
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(); fn(); e1.record()
-            torch.cuda.synchronize()
-            tot += e0.elapsed_time(e1)
-        return tot / iters
-
-    rows = []
-    for T in sorted(PAPER_TP8_MS):
-        q, k, v, d_o = cowa_inputs.make_train_inputs(11, 1, T, Hq_r, 1, D, device=dev)
-        o = torch.empty_like(q)
-        lse = torch.empty((1, Hq_r, T), dtype=torch.float32, device=dev)
-        dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
-        qd, od = q[:, :, -1].contiguous(), torch.empty((1, Hq_r, D), dtype=torch.bfloat16, device=dev)
-        lsed = torch.empty((1, Hq_r), dtype=torch.float32, device=dev)
-        lens = torch.tensor([T], dtype=torch.int32, device=dev)
-        worst = {}
-        for layout in ("cowa", "eq", "full"):  # default equal-width bands, equal-area bands, dense
-            for r in range(rank, TP, world):
-                if layout == "eq":
-                    p = cowa.make_params(windows=cowa.cowa_equal_area_windows(T, T, TP, r, 1, sink, near),
-                                         softmax_scale=scale)
-                else:
-                    p = cowa.make_params(sink=sink, local=near, softmax_scale=scale, full_attn=(layout == "full"),
-                                         hkv_global=TP, hkv_offset=r)
-                ws = torch.empty(max(cowa.cowa_bwd_workspace_bytes(1, T, Hq_r, 1, D, p), 16), dtype=torch.uint8,
-                                 device=dev)
-                wsd = torch.empty(max(cowa.cowa_decode_workspace_bytes(1, T, Hq_r, 1, D, p), 16), dtype=torch.uint8,
-                                  device=dev)
-                t = {"fwd": timed(lambda: cowa.cowa_fwd(q, k, v, o, lse, p)),
-                     "bwd": timed(lambda: cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, p, ws))}
-                if layout != "eq":  # decode keeps the equal-width rule (Sec. 2.1), so there is no third variant
-                    t["dec"] = timed(lambda: cowa.cowa_decode(qd, k, v, lens, od, lsed, p, wsd))
-                for ph, ms in t.items():
-                    key = layout + "_" + ph
-                    worst[key] = max(worst.get(key, 0.0), ms)
-                if layout == "full":
-                    break  # dense shards are identical on every rank
-        cowa.cowa_check_device_status()
-        worst = {k_: max_over_ranks(v_, world) for k_, v_ in sorted(worst.items())}
-        pf, pc, pfb, pcb, pfd, pcd = PAPER_TP8_MS[T]
-        rows.append({"T": T, **{k_ + "_ms": v_ for k_, v_ in worst.items()},
-                     "speedup_fwd": worst["full_fwd"] / worst["cowa_fwd"],
-                     "speedup_bwd": worst["full_bwd"] / worst["cowa_bwd"],
-                     "speedup_fwd_equal_area": worst["full_fwd"] / worst["eq_fwd"],
-                     "speedup_bwd_equal_area": worst["full_bwd"] / worst["eq_bwd"],
-                     "speedup_dec": worst["full_dec"] / worst["cowa_dec"],
-                     "paper_h100_ms": {"full_fwd": pf, "cowa_fwd": pc, "full_bwd": pfb, "cowa_bwd": pcb,
-                                       "full_dec": pfd, "cowa_dec": pcd}})
-        del q, k, v, d_o, o, lse, dq, dk, dv
+    iters, warm = max(args.steps, 3), max(args.warmup, 3)
+    rows = reduce_worst(tp_replica_rows(cowa, cowa_inputs, dev, sorted(PAPER_TP8_MS), rank, world, warm, iters), world)
+    for r in rows:
+        pf, pc, pfb, pcb, pfd, pcd = PAPER_TP8_MS[r["T"]]
+        r.update({"speedup_fwd": r["full_fwd_ms"] / r["cowa_fwd_ms"], "speedup_bwd": r["full_bwd_ms"] / r["cowa_bwd_ms"],
+                  "speedup_fwd_equal_area": r["full_fwd_ms"] / r["eq_fwd_ms"],
+                  "speedup_bwd_equal_area": r["full_bwd_ms"] / r["eq_bwd_ms"],
+                  "speedup_dec": r["full_dec_ms"] / r["cowa_dec_ms"],
+                  "paper_h100_ms": {"full_fwd": pf, "cowa_fwd": pc, "full_bwd": pfb, "cowa_bwd": pcb,
+                                    "full_dec": pfd, "cowa_dec": pcd}})
     if rank != 0:
         return
     last = rows[-1]
     print(json.dumps({
         "metric": "cowa_tp8_shard_fwd_bwd_ms_128k", "value": last["cowa_fwd_ms"] + last["cowa_bwd_ms"], "unit": "ms",
-        "n_gpus": world, "steps": iters, "warmup": max(args.warmup, 3), "higher_is_better": False,
+        "n_gpus": world, "steps": iters, "warmup": warm, "higher_is_better": False,
         "scaling": "strong", "vs_baseline": (last["cowa_fwd_ms"] + last["cowa_bwd_ms"]) / (21.758 + 51.509),
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": "TP=8 shards of B=1, Hq=64, Hkv=8, D=128, sink+near=128+896, T=1K..128K",
-                   "shards_per_gpu": TP // world if world <= TP else 1, "l2": "flushed before every timed call",
+                   "shards_per_gpu": 8 // world if world <= 8 else 1, "l2": "flushed before every timed call",
                    "latency": "slowest shard (max over the 8 ranks' launches)"},
         "rows": rows}))
 
@@ -741,8 +847,12 @@ def main():
     ap.add_argument("--tp-replica", action="store_true",
                     help="time the TP=8 shards of the paper's operator benchmark shape instead of the default step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-table", action="store_true",
+                    help="skip the rows of the other configurations (tiny, 8K, 8K control, 32K) and the TP=8 shard row")
+    ap.add_argument("--windows", default="default", choices=["default", "dup1", "dup2"],
+                    help="dup<m>: duplicated-window control, the first m bands repeated over the KV heads")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
-    ap.add_argument("--train-cfg", default=TRAIN_CFG, choices=["8k", "32k", "128k"],
+    ap.add_argument("--train-cfg", default=TRAIN_CFG, choices=["tiny", "8k", "32k", "128k"],
                     help="training configuration (default: the 128K headline; smaller ones are for profiling)")
     ap.add_argument("--decode-batch", type=int, default=0, help="override the decode batch (profiling)")
     ap.add_argument("--deterministic", action="store_true",

@@ -15,12 +15,15 @@
  *   - q, k, v, o, d_o, dq, dk, dv are bf16; lse and workspaces are fp32/bytes.
  *   - Default layout is contiguous head-major [B, H, T, D] with D innermost
  *     (Algorithm 1/2 REQUIRE lines, plus a batch axis).  Base pointers must be
- *     16-byte aligned.
+ *     16-byte aligned.  Other layouts of the batched calls are described by element
+ *     strides in cowa_params_t (D always contiguous): e.g. a [B, T, H, D] projection
+ *     output or a [B, Tmax, Hkv, D] cache is passed without a copy.
  *   - lse is the natural-log logsumexp of softmax_scale * q.k over the visible keys
  *     (Algorithm 1 line 17), fp32 [B, Hq, T].
  *   - The caller owns every buffer, workspaces included.  The library allocates no
  *     device memory and keeps no state between calls except cached kernel
- *     attributes.  All work is enqueued on `stream`; no call synchronises.
+ *     attributes and the per-thread error code behind cowa_last_cuda_error().
+ *     All work is enqueued on `stream`; no call synchronises.
  *   - Return value: COWA_OK (0) or a negative cowa_status_t.  Arguments are validated
  *     before anything is launched.  There is no CPU fallback.
  *   - Preconditions not checked on the device: near >= 1 for every head (so each
@@ -39,14 +42,18 @@ extern "C" {
 typedef enum {
   COWA_OK = 0,
   COWA_ERR_INVALID_ARG = -1,        /* null pointer, non-positive size, Hq % Hkv != 0, bad window */
-  COWA_ERR_UNSUPPORTED = -2,        /* D not in {64,128}; strides other than contiguous */
-  COWA_ERR_MISALIGNED = -3,         /* a base pointer is not 16-byte aligned */
+  COWA_ERR_UNSUPPORTED = -2,        /* D not in {64,128}; strides given to a call that takes none */
+  COWA_ERR_MISALIGNED = -3,         /* a base pointer is not 16-byte aligned, or a stride is not a multiple of
+                                       8 elements (16 bytes) */
   COWA_ERR_WORKSPACE_TOO_SMALL = -4,
   COWA_ERR_CUDA = -5,               /* a CUDA call failed; see cowa_last_cuda_error() */
   COWA_ERR_DEVICE_TIMEOUT = -6,     /* reported by cowa_check_device_status(): a bounded device wait ran out */
   COWA_ERR_STATIC_SCRATCH_EXCEEDED = -7, /* cowa_decode_static: the call needs more scratch than the built-in array holds */
-  COWA_ERR_DEVICE_BAD_SEQLENS = -8  /* reported by cowa_check_device_status(): cowa_prefill_varlen met a sequence
+  COWA_ERR_DEVICE_BAD_SEQLENS = -8, /* reported by cowa_check_device_status(): cowa_prefill_varlen met a sequence
                                        with N_q > N_k in its device-side offset arrays and skipped it */
+  COWA_ERR_DEVICE_DQ_RANGE = -9     /* reported by cowa_check_device_status(): a backward call with
+                                       deterministic = 1 met a dQ partial sum outside the fixed-point range
+                                       (|x| >= 8192), or a final |dQ| >= 4096; its dq is not to be trusted */
 } cowa_status_t;
 
 /* One KV head's windows: the paper's 4-tuple (sink width, near width, gap after the
@@ -70,7 +77,24 @@ typedef struct {
                             blocks arrive (Algorithm 2 line 15's AtomicAdd; results vary in the last bits
                             from run to run).  1: the partial sums are added as 32-bit fixed point with
                             18 fractional bits, which is exact and order-independent, so dQ is bitwise
-                            reproducible; requires |dQ| < 8192 and rounds each partial to 2^-19. */
+                            reproducible; requires |dQ| < 8192 and rounds each partial to 2^-19.  A partial
+                            sum of one tile that leaves that range, or a final |dQ| >= 4096 (half of it: a
+                            wrapped total lands there in most cases), sets a device flag that
+                            cowa_check_device_status() returns as COWA_ERR_DEVICE_DQ_RANGE. */
+  /* Element strides (batch, head, token) of q, k, v, o; the D axis is contiguous.  All three zero (the
+   * default) means contiguous head-major [B, H, T, D].  Otherwise every stride must be a non-negative multiple
+   * of 8 elements and the token stride at least D.  Used by cowa_fwd, cowa_prefill, cowa_bwd, cowa_bwd_prefill
+   * (there d_o is laid out like o, dq like q, dk like k, dv like v) and by cowa_decode / cowa_decode_static
+   * (k_strides, v_strides describe the cache; q and o stay [B, Hq, D]).  The packed (varlen), multi-token and
+   * paged calls take contiguous tensors only and return COWA_ERR_UNSUPPORTED when a stride is set.  lse is
+   * always contiguous. */
+  int64_t q_strides[3], k_strides[3], v_strides[3], o_strides[3];
+  /* cowa_bwd / cowa_bwd_prefill / cowa_bwd_varlen only: optional CUDA events (cudaEvent_t handles owned by the
+   * caller, or NULL) recorded on the call's stream just before and just after the main backward kernel
+   * (Algorithm 2's loops), so that a profiler can time that kernel apart from the preprocess, memset and
+   * conversion launches of the same call. */
+  void* bwd_main_start_event;
+  void* bwd_main_stop_event;
 } cowa_params_t;
 
 /* Training / prefill forward, Algorithm 1.  N_q = N_k = T.
@@ -118,12 +142,6 @@ int cowa_bwd(const void* q, const void* k, const void* v, const void* o, const f
              const void* d_o, void* dq, void* dk, void* dv,
              int B, int T, int Hq, int Hkv, int D, const cowa_params_t* p,
              void* workspace, size_t workspace_bytes, void* stream);
-
-/* Profiling hook (no counterpart in the paper).  cowa_bwd enqueues a memset, a preprocess kernel, the
- * main kernel (Algorithm 2's loops) and a dQ conversion kernel.  After this call, every cowa_bwd issued
- * from the same host thread records `start_event` just before and `stop_event` just after the main kernel
- * on the call's stream (both are cudaEvent_t handles owned by the caller; NULL, NULL switches it off). */
-int cowa_bwd_set_profile_events(void* start_event, void* stop_event);
 
 /* Backward of cowa_prefill: the same Algorithm 2 with N_q <= N_k (queries bottom-right aligned, Eq.
  * fwa_distance; windows from N_k).  q, o, d_o, dq [B,Hq,Nq,D]; k, v, dk, dv [B,Hkv,Nk,D]; lse [B,Hq,Nq].
@@ -257,10 +275,17 @@ int cowa_schedule_dump(int which, int Nq, int Nk, int Hkv, const cowa_params_t* 
 int cowa_tile_counts(int Nq, int Nk, int Hkv, const cowa_params_t* p, int64_t out[3]);
 
 /* The kernels bound every device-side wait; a wait that runs out sets a flag in a device word
- * instead of hanging.  This call synchronises `stream`, reads and clears the flag, and returns
- * COWA_OK, COWA_ERR_DEVICE_TIMEOUT or COWA_ERR_DEVICE_BAD_SEQLENS (COWA_ERR_CUDA if the stream itself
- * reports an error). */
+ * instead of hanging.  This call synchronises `stream`, reads and clears the flags, and returns
+ * COWA_OK, COWA_ERR_DEVICE_TIMEOUT, COWA_ERR_DEVICE_BAD_SEQLENS or COWA_ERR_DEVICE_DQ_RANGE, in that
+ * order of precedence when several are set (COWA_ERR_CUDA if the stream itself reports an error). */
 int cowa_check_device_status(void* stream);
+
+/* Self-test of the bounded waits (no counterpart in the paper).  Enqueues a one-block kernel that waits,
+ * with the same wait routine the training kernels use but a limit of `limit_clocks` SM clocks (clamped to
+ * [2^10, 2^24]), on a barrier that nothing ever arrives at.  The wait must give up, set the timeout flag
+ * and let the kernel end normally: the next cowa_check_device_status() then returns
+ * COWA_ERR_DEVICE_TIMEOUT once.  Nothing else is touched. */
+int cowa_selftest_bounded_wait(long long limit_clocks, void* stream);
 
 const char* cowa_status_string(int status);
 /* cudaError_t value of the most recent failing CUDA call made by this library on this thread. */

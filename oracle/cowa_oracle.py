@@ -110,24 +110,26 @@ def kv_head_of(h, h_q, h_k):
 # --------------------------------------------------------------------------
 
 
-def causal_distance(n_q, n_k, rows=None):
-    """delta[i_q, i_k] = i_q + (N_k - N_q) - i_k  (bottom-right aligned)."""
+def causal_distance(n_q, n_k, rows=None, cols=None):
+    """delta[i_q, i_k] = i_q + (N_k - N_q) - i_k  (bottom-right aligned), for the given query rows and key
+    columns (all of them by default)."""
     # int32 holds every distance for sequences below 2^30 tokens
     it = np.int32 if max(int(n_q), int(n_k)) < (1 << 30) else np.int64
     rows = np.arange(n_q, dtype=it) if rows is None else np.asarray(rows, dtype=it)
-    i_k = np.arange(n_k, dtype=it)
+    i_k = np.arange(n_k, dtype=it) if cols is None else np.asarray(cols, dtype=it)
     return rows[:, None] + it(int(n_k) - int(n_q)) - i_k[None, :]
 
 
-def visible_mask(n_q, n_k, window, rows=None):
-    """Boolean [len(rows), N_k]: key visible to the query under one head's tuple.
+def visible_mask(n_q, n_k, window, rows=None, cols=None):
+    """Boolean [len(rows), len(cols)] (all N_k keys by default): key visible to the query under one head's
+    tuple.
 
     near: 0 <= delta < near;  sink: i_k < sink and delta >= 0;
     long: near + gap <= delta < near + gap + long.  Union of the three.
     """
     w_sink, w_near, gap, w_long = (int(x) for x in window)
-    delta = causal_distance(n_q, n_k, rows)
-    i_k = np.arange(n_k, dtype=delta.dtype)[None, :]
+    delta = causal_distance(n_q, n_k, rows, cols)
+    i_k = (np.arange(n_k, dtype=delta.dtype) if cols is None else np.asarray(cols, dtype=delta.dtype))[None, :]
     near = (delta >= 0) & (delta < w_near)
     sink = (i_k < w_sink) & (delta >= 0)
     far = (delta >= w_near + gap) & (delta < w_near + gap + w_long)
@@ -268,13 +270,14 @@ def backward_dkdv_cols(q, k, v, d_o, windows, scale, hk, cols, row_block=1024):
     vc_sel = np.asarray(v[hk][cols], dtype=np.float64)
     for r0 in range(0, n_q, row_block):
         rows = np.arange(r0, min(r0 + row_block, n_q))
-        mask = visible_mask(n_q, n_k, windows[hk], rows)
-        sel = mask[:, cols]
+        # rows that see none of the selected columns contribute nothing: find them from the mask on those
+        # columns alone before the mask over all keys is built for the rest
+        sel = visible_mask(n_q, n_k, windows[hk], rows, cols)
         live = np.flatnonzero(sel.any(axis=1))
         if len(live) == 0:
             continue
         rows = rows[live]
-        mask = mask[live]
+        mask = visible_mask(n_q, n_k, windows[hk], rows)
         keep = mask.any(axis=0)
         keep[cols] = True  # selected columns stay addressable even if unseen here
         allc = np.flatnonzero(keep)

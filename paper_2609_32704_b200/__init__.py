@@ -8,7 +8,8 @@ from .binding import (  # noqa: F401
     cowa_fwd, cowa_prefill, cowa_prefill_varlen, cowa_bwd, cowa_decode, cowa_decode_multi, cowa_decode_paged, cowa_decode_multi_workspace_bytes,
     cowa_decode_static, cowa_decode_static_capacity,
     cowa_bwd_workspace_bytes, cowa_bwd_varlen, cowa_bwd_varlen_workspace_bytes,
-    cowa_bwd_prefill, cowa_bwd_prefill_workspace_bytes, cowa_bwd_set_profile_events, cowa_decode_workspace_bytes,
+    cowa_bwd_prefill, cowa_bwd_prefill_workspace_bytes, with_bwd_events, cowa_decode_workspace_bytes,
     cowa_default_windows, cowa_equal_area_windows, cowa_schedule_dump, cowa_tile_counts, cowa_check_device_status,
+    cowa_selftest_bounded_wait,
     cowa_status_string, SCHED_FWD, SCHED_BWD, SCHED_DECODE,
 )

@@ -31,6 +31,9 @@ class Params(C.Structure):
         ("sink", C.c_int32), ("local", C.c_int32), ("block_q", C.c_int32), ("block_k", C.c_int32),
         ("hkv_global", C.c_int32), ("hkv_offset", C.c_int32), ("windows", C.POINTER(Window)),
         ("full_attn", C.c_int32), ("softmax_scale", C.c_float), ("deterministic", C.c_int32),
+        ("q_strides", C.c_int64 * 3), ("k_strides", C.c_int64 * 3), ("v_strides", C.c_int64 * 3),
+        ("o_strides", C.c_int64 * 3),
+        ("bwd_main_start_event", C.c_void_p), ("bwd_main_stop_event", C.c_void_p),
     ]
 
 
@@ -74,8 +77,6 @@ def lib():
         L.cowa_decode_multi_workspace_bytes.restype = sz
         L.cowa_decode_static_capacity.argtypes = []
         L.cowa_decode_static_capacity.restype = sz
-        L.cowa_bwd_set_profile_events.argtypes = [vp, vp]
-        L.cowa_bwd_set_profile_events.restype = i32
         L.cowa_bwd_workspace_bytes.argtypes = [i32] * 5 + [pp]
         L.cowa_bwd_workspace_bytes.restype = sz
         L.cowa_decode_workspace_bytes.argtypes = [i32] * 5 + [pp]
@@ -90,6 +91,8 @@ def lib():
         L.cowa_tile_counts.restype = i32
         L.cowa_check_device_status.argtypes = [vp]
         L.cowa_check_device_status.restype = i32
+        L.cowa_selftest_bounded_wait.argtypes = [C.c_longlong, vp]
+        L.cowa_selftest_bounded_wait.restype = i32
         L.cowa_status_string.argtypes = [i32]
         L.cowa_status_string.restype = C.c_char_p
         L.cowa_last_cuda_error.argtypes = []
@@ -130,20 +133,61 @@ def _ptr(t):
     return C.c_void_p(0 if t is None else t.data_ptr())
 
 
-def _need(t, dtype, name):
+def _need(t, dtype, name, strided=False):
+    """Contiguous CUDA tensor of `dtype`; with strided=True any batch / head / token strides are accepted as
+    long as the last axis is contiguous (the strides then travel in cowa_params_t)."""
     import torch
-    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous() and t.dtype == dtype):
-        raise TypeError(f"{name}: expected a contiguous CUDA tensor of {dtype}")
+    ok = isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == dtype
+    if ok and strided:
+        ok = t.stride(-1) == 1 or t.shape[-1] == 1
+    elif ok:
+        ok = t.is_contiguous()
+    if not ok:
+        kind = "CUDA tensor with a contiguous last axis" if strided else "contiguous CUDA tensor"
+        raise TypeError(f"{name}: expected a {kind} of {dtype}")
+
+
+def _copy_params(params):
+    p = Params.from_buffer_copy(params)
+    p._keepalive = params  # the windows array (if any) lives as long as the original
+    return p
+
+
+def _with_strides(params, **tensors):
+    """`params` itself when every tensor is contiguous, else a copy whose <name>_strides hold the tensors'
+    (batch, head, token) element strides."""
+    if all(t.is_contiguous() for t in tensors.values()):
+        return params
+    p = _copy_params(params)
+    for name, t in tensors.items():
+        getattr(p, name + "_strides")[:] = [t.stride(0), t.stride(1), t.stride(2)]
+    return p
+
+
+def with_bwd_events(params, start_event, stop_event):
+    """Copy of `params` that makes cowa_bwd record the two torch.cuda.Event objects (already created, e.g.
+    recorded once) just before and after its main kernel."""
+    p = _copy_params(params)
+    p.bwd_main_start_event = start_event.cuda_event
+    p.bwd_main_stop_event = stop_event.cuda_event
+    return p
+
+
+def _same_layout(a, b, na, nb):
+    if a.shape != b.shape or a.stride() != b.stride():
+        raise TypeError(f"{na} must have the shape and strides of {nb}")
 
 
 def cowa_fwd(q, k, v, o, lse, params):
-    """q [B,Hq,T,D], k/v [B,Hkv,T,D] bf16 -> o (bf16), lse (fp32 [B,Hq,T]); all preallocated."""
+    """q [B,Hq,T,D], k/v [B,Hkv,T,D] bf16 -> o (bf16), lse (fp32 [B,Hq,T]); all preallocated.  q, k, v, o may
+    be strided views with that shape (e.g. x.transpose(1, 2) of a [B,T,H,D] tensor)."""
     import torch
     for t, n in ((q, "q"), (k, "k"), (v, "v"), (o, "o")):
-        _need(t, torch.bfloat16, n)
+        _need(t, torch.bfloat16, n, strided=True)
     _need(lse, torch.float32, "lse")
     B, Hq, T, D = q.shape
     Hkv = k.shape[1]
+    params = _with_strides(params, q=q, k=k, v=v, o=o)
     _check(lib().cowa_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), B, T, Hq, Hkv, D,
                           C.byref(params), _stream()), "cowa_fwd")
 
@@ -152,10 +196,11 @@ def cowa_prefill(q, k, v, o, lse, params):
     """Forward with N_q <= N_k (bottom-right aligned): q [B,Hq,Nq,D], k/v [B,Hkv,Nk,D] -> o, lse [B,Hq,Nq]."""
     import torch
     for t, n in ((q, "q"), (k, "k"), (v, "v"), (o, "o")):
-        _need(t, torch.bfloat16, n)
+        _need(t, torch.bfloat16, n, strided=True)
     _need(lse, torch.float32, "lse")
     B, Hq, Nq, D = q.shape
     Hkv, Nk = k.shape[1], k.shape[2]
+    params = _with_strides(params, q=q, k=k, v=v, o=o)
     _check(lib().cowa_prefill(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), B, Nq, Nk, Hq, Hkv, D,
                               C.byref(params), _stream()), "cowa_prefill")
 
@@ -184,13 +229,17 @@ def cowa_bwd_workspace_bytes(B, T, Hq, Hkv, D, params):
 
 
 def cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, params, workspace):
-    """Gradients dq, dk, dv (bf16, preallocated) of cowa_fwd; workspace: uint8 CUDA tensor."""
+    """Gradients dq, dk, dv (bf16, preallocated) of cowa_fwd; workspace: uint8 CUDA tensor.  Strided views are
+    accepted when d_o is laid out like o, dq like q, dk like k and dv like v."""
     import torch
     for t, n in ((q, "q"), (k, "k"), (v, "v"), (o, "o"), (d_o, "d_o"), (dq, "dq"), (dk, "dk"), (dv, "dv")):
-        _need(t, torch.bfloat16, n)
+        _need(t, torch.bfloat16, n, strided=True)
     _need(lse, torch.float32, "lse")
+    for a_, b_, na, nb in ((d_o, o, "d_o", "o"), (dq, q, "dq", "q"), (dk, k, "dk", "k"), (dv, v, "dv", "v")):
+        _same_layout(a_, b_, na, nb)
     B, Hq, T, D = q.shape
     Hkv = k.shape[1]
+    params = _with_strides(params, q=q, k=k, v=v, o=o)
     _check(lib().cowa_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(d_o), _ptr(dq), _ptr(dk),
                           _ptr(dv), B, T, Hq, Hkv, D, C.byref(params), _ptr(workspace),
                           workspace.numel() * workspace.element_size(), _stream()), "cowa_bwd")
@@ -204,10 +253,13 @@ def cowa_bwd_prefill(q, k, v, o, lse, d_o, dq, dk, dv, params, workspace):
     """Backward with N_q <= N_k: q/o/d_o/dq [B,Hq,Nq,D], k/v/dk/dv [B,Hkv,Nk,D], lse [B,Hq,Nq]."""
     import torch
     for t, n in ((q, "q"), (k, "k"), (v, "v"), (o, "o"), (d_o, "d_o"), (dq, "dq"), (dk, "dk"), (dv, "dv")):
-        _need(t, torch.bfloat16, n)
+        _need(t, torch.bfloat16, n, strided=True)
     _need(lse, torch.float32, "lse")
+    for a_, b_, na, nb in ((d_o, o, "d_o", "o"), (dq, q, "dq", "q"), (dk, k, "dk", "k"), (dv, v, "dv", "v")):
+        _same_layout(a_, b_, na, nb)
     B, Hq, Nq, D = q.shape
     Hkv, Nk = k.shape[1], k.shape[2]
+    params = _with_strides(params, q=q, k=k, v=v, o=o)
     _check(lib().cowa_bwd_prefill(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(d_o), _ptr(dq), _ptr(dk),
                                   _ptr(dv), B, Nq, Nk, Hq, Hkv, D, C.byref(params), _ptr(workspace),
                                   workspace.numel() * workspace.element_size(), _stream()), "cowa_bwd_prefill")
@@ -233,27 +285,24 @@ def cowa_bwd_varlen(q, k, v, o, lse, d_o, dq, dk, dv, cu_seqlens, params, worksp
                                  workspace.numel() * workspace.element_size(), _stream()), "cowa_bwd_varlen")
 
 
-def cowa_bwd_set_profile_events(start_event, stop_event):
-    """torch.cuda.Event pair (already created, e.g. recorded once) to be recorded around the main
-    backward kernel of the following cowa_bwd calls; (None, None) switches the hook off."""
-    h = lambda e: C.c_void_p(0 if e is None else e.cuda_event)
-    _check(lib().cowa_bwd_set_profile_events(h(start_event), h(stop_event)), "cowa_bwd_set_profile_events")
-
-
 def cowa_decode_workspace_bytes(B, Tmax, Hq, Hkv, D, params):
     return int(lib().cowa_decode_workspace_bytes(B, Tmax, Hq, Hkv, D, C.byref(params)))
 
 
 def cowa_decode(q, kcache, vcache, lens, o, lse, params, workspace):
-    """q [B,Hq,D], caches [B,Hkv,Tmax,D] bf16, lens int32 [B] (device) -> o [B,Hq,D], lse [B,Hq] or None."""
+    """q [B,Hq,D], caches [B,Hkv,Tmax,D] bf16 (strided views with that shape are accepted, e.g. a
+    [B,Tmax,Hkv,D] cache transposed), lens int32 [B] (device) -> o [B,Hq,D], lse [B,Hq] or None."""
     import torch
-    for t, n in ((q, "q"), (kcache, "kcache"), (vcache, "vcache"), (o, "o")):
+    for t, n in ((q, "q"), (o, "o")):
         _need(t, torch.bfloat16, n)
+    for t, n in ((kcache, "kcache"), (vcache, "vcache")):
+        _need(t, torch.bfloat16, n, strided=True)
     _need(lens, torch.int32, "lens")
     if lse is not None:
         _need(lse, torch.float32, "lse")
     B, Hq, D = q.shape
     Hkv, Tmax = kcache.shape[1], kcache.shape[2]
+    params = _with_strides(params, k=kcache, v=vcache)
     _check(lib().cowa_decode(_ptr(q), _ptr(kcache), _ptr(vcache), _ptr(lens), _ptr(o), _ptr(lse), B, Tmax,
                              Hq, Hkv, D, C.byref(params), _ptr(workspace),
                              workspace.numel() * workspace.element_size(), _stream()), "cowa_decode")
@@ -351,6 +400,11 @@ def cowa_tile_counts(Nq, Nk, Hkv, params):
 
 def cowa_check_device_status():
     _check(lib().cowa_check_device_status(_stream()), "cowa_check_device_status")
+
+
+def cowa_selftest_bounded_wait(limit_clocks=1 << 20):
+    """Enqueues the library's self-test kernel whose bounded wait must run out (see cowa.h)."""
+    _check(lib().cowa_selftest_bounded_wait(int(limit_clocks), _stream()), "cowa_selftest_bounded_wait")
 
 
 def cowa_status_string(status):

@@ -5,10 +5,21 @@
 #include <algorithm>
 #include <vector>
 #include "cowa_common.h"
+#include "cowa_ptx.cuh"
 
 namespace {
 thread_local int g_last_cuda_error = 0;
 __device__ unsigned int g_cowa_status_word = 0;
+
+// One warp-free block: thread 0 waits on a barrier that has no arrivals until the bounded wait gives up.
+__global__ void cowa_selftest_wait_kernel(unsigned int* status, long long limit) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    cowa_ptx::mbar_init(&bar, 1);
+    cowa_ptx::fence_mbar_init();
+    cowa_ptx::mbar_wait(&bar, 0, status, limit);
+  }
+}
 }  // namespace
 
 namespace cowa {
@@ -32,6 +43,23 @@ unsigned int* device_status_word() {
   return cache[dev];
 }
 
+int resolve_strides(const int64_t s[3], int H, long long T, int D, CowaStrides* out) {
+  if (s[0] == 0 && s[1] == 0 && s[2] == 0) {
+    out->t = D; out->h = (long long)T * D; out->b = (long long)H * T * D;
+    return COWA_OK;
+  }
+  if (s[0] < 0 || s[1] < 0 || s[2] < D) return COWA_ERR_INVALID_ARG;
+  if ((s[0] | s[1] | s[2]) & 7) return COWA_ERR_MISALIGNED;
+  out->b = s[0]; out->h = s[1]; out->t = s[2];
+  return COWA_OK;
+}
+
+bool any_stride_set(const cowa_params_t* p) {
+  for (int i = 0; i < 3; ++i)
+    if (p->q_strides[i] || p->k_strides[i] || p->v_strides[i] || p->o_strides[i]) return true;
+  return false;
+}
+
 int resolve_windows(int Nk, int Hkv, const cowa_params_t* p, CowaHeadWindows* out) {
   if (!p || Hkv <= 0 || Nk <= 0) return COWA_ERR_INVALID_ARG;
   if (Hkv > COWA_MAX_HKV) return COWA_ERR_UNSUPPORTED;
@@ -44,7 +72,9 @@ int resolve_windows(int Nk, int Hkv, const cowa_params_t* p, CowaHeadWindows* ou
     } else if (p->windows) {
       const cowa_window_t& t = p->windows[h];
       if (t.sink < 0 || t.near < 1 || t.gap < 0 || t.len < 0) return COWA_ERR_INVALID_ARG;
-      w.s = t.sink; w.n = t.near; w.g = t.gap; w.l = t.len;
+      // no key lies further than Nk away: widths beyond Nk mean the same as Nk, and clamping them keeps the
+      // sums near + gap + len inside 32 bits everywhere
+      w.s = std::min(t.sink, Nk); w.n = std::min(t.near, Nk); w.g = std::min(t.gap, Nk); w.l = std::min(t.len, Nk);
     } else {
       if (p->sink < 0 || p->local < 1) return COWA_ERR_INVALID_ARG;
       w = cowa_default_window(Nk, hg, p->hkv_offset + h, p->sink, p->local);
@@ -198,8 +228,19 @@ int cowa_check_device_status(void* stream) {
   if (host != 0) {
     COWA_CUDA_TRY(cudaMemsetAsync(word, 0, sizeof(host), s));
     COWA_CUDA_TRY(cudaStreamSynchronize(s));
-    return (host & 1u) ? COWA_ERR_DEVICE_TIMEOUT : COWA_ERR_DEVICE_BAD_SEQLENS;
+    if (host & COWA_DEV_TIMEOUT) return COWA_ERR_DEVICE_TIMEOUT;
+    if (host & COWA_DEV_BAD_SEQLENS) return COWA_ERR_DEVICE_BAD_SEQLENS;
+    return COWA_ERR_DEVICE_DQ_RANGE;
   }
+  return COWA_OK;
+}
+
+int cowa_selftest_bounded_wait(long long limit_clocks, void* stream) {
+  unsigned int* word = cowa::device_status_word();
+  if (!word) return COWA_ERR_CUDA;
+  const long long limit = std::min(std::max(limit_clocks, 1ll << 10), 1ll << 24);
+  cowa_selftest_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(word, limit);
+  COWA_CUDA_TRY(cudaGetLastError());
   return COWA_OK;
 }
 
@@ -216,6 +257,8 @@ const char* cowa_status_string(int status) {
       return "cowa_decode_static: the call needs more scratch than the library's built-in array holds";
     case COWA_ERR_DEVICE_BAD_SEQLENS:
       return "cowa_prefill_varlen: a sequence with N_q > N_k was skipped";
+    case COWA_ERR_DEVICE_DQ_RANGE:
+      return "deterministic backward: a dQ value left the fixed-point range";
     default: return "unknown status";
   }
 }

@@ -16,9 +16,10 @@
 //                   atomics (Algorithm 2 line 17 needs them only because it gives each QO head its
 //                   own program).  dQ^T is drained by a separate warpgroup through shared memory and
 //                   added to the fp32 accumulator with TMA bulk reductions (Algorithm 2 line 15).
-//                   Warp roles: TMA producer / MMA issuer / two compute warpgroups (P, dS; 32 query
-//                   columns each) / dQ drain warpgroup, connected by mbarriers; S^T is double
-//                   buffered so that the MMAs of steps n+1, n+2 overlap the element-wise work of
+//                   Warp roles: TMA producer / MMA issuer / two compute warpgroups (P, dS; each takes 32
+//                   of the 64 query columns of every step, which halves the latency between S^T and
+//                   dS^T) / dQ drain warpgroup, connected by mbarriers; S^T is double buffered so that the
+//                   MMAs of steps n+1, n+2 overlap the element-wise work of
 //                   step n.  Blocks are ordered sink tiles first (they meet every query tile), then
 //                   head by head with ascending KV tile, so that the blocks in flight sweep the same
 //                   dQ rows at nearly the same time and the reductions hit in L2.
@@ -131,8 +132,8 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   uint64_t* bar_ld_empty = bars + 1 + NST;      // [NST]  the step's products have consumed the stage
   uint64_t* bar_s_full = bars + 1 + 2 * NST;    // [2]    S^T of a step is in TMEM buffer b
   uint64_t* bar_dp_full = bars + 3 + 2 * NST;   // [2]    dP^T ...
-  uint64_t* bar_p_ready = bars + 5 + 2 * NST;   // [2]    count 128: P^T written over S^T
-  uint64_t* bar_ds_ready = bars + 7 + 2 * NST;  // [2]    count 128: dS^T in TMEM and shared memory, dP^T consumed
+  uint64_t* bar_p_ready = bars + 5 + 2 * NST;   // [2]    count 256: P^T written over S^T
+  uint64_t* bar_ds_ready = bars + 7 + 2 * NST;  // [2]    count 256: dS^T in TMEM and shared memory, dP^T consumed
   uint64_t* bar_dq_full = bars + 9 + 2 * NST;   // [2]    dQ^T is in the columns dP^T left
   uint64_t* bar_dq_free = bars + 11 + 2 * NST;  // [2]    count 128: dQ^T drained
   uint64_t* bar_done = bars + 13 + 2 * NST;
@@ -178,7 +179,7 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     rbase = a.cu[b];
     Nq = Nk = a.cu[b + 1] - rbase;
     if (rbase < 0 || rbase + Nk > a.total) {  // malformed offsets: report, touch nothing
-      if (threadIdx.x == 0) atomicOr(a.status, 2u);
+      if (threadIdx.x == 0) atomicOr(a.status, (unsigned)COWA_DEV_BAD_SEQLENS);
       return;
     }
     w = a.wins.w[hk];
@@ -192,8 +193,10 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const int cnt = cowa_range_len(rg[0]) + cowa_range_len(rg[1]);  // QO steps per head
   const int gs = a.G / a.parts;          // heads of the group handled by this block
   const int N = cnt * gs;
-  const int bhk = VARLEN ? hk : b * a.Hkv + hk;                                     // third TMA coordinate of K, V, dK, dV
-  const int bhq0 = (VARLEN ? 0 : b * a.Hq) + hk * a.G + part * gs;                  // ... of Q, dO, dQ: first head of this block
+  const int bt = VARLEN ? 0 : b;                                                    // batch coordinate of the tensor maps
+  const int bhk = VARLEN ? hk : b * a.Hkv + hk;                                     // (batch, KV head) row of the partial dK, dV slots
+  const int hq0 = hk * a.G + part * gs;                                             // first QO head of this block
+  const int bhq0 = (VARLEN ? 0 : b * a.Hq) + hq0;                                   // ... as a row of lse2 / delta / dq_acc
   const size_t vec_stride = (size_t)a.Tpad;                                         // rows per head in lse2 / delta / dq_acc
   const bool tail_kv = VARLEN && (k0 + BKV > Nk);  // rows after the tile's last valid one belong to the next sequence
 
@@ -202,7 +205,7 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     for (int s = 0; s < NST; ++s) { mbar_init(bar_ld_full + s, 1); mbar_init(bar_ld_empty + s, 1); }
     for (int s = 0; s < 2; ++s) {
       mbar_init(bar_s_full + s, 1); mbar_init(bar_dp_full + s, 1);
-      mbar_init(bar_p_ready + s, 128); mbar_init(bar_ds_ready + s, 128);
+      mbar_init(bar_p_ready + s, 256); mbar_init(bar_ds_ready + s, 256);
       mbar_init(bar_dq_full + s, 1); mbar_init(bar_dq_free + s, 128);
     }
     mbar_init(bar_done, 1);
@@ -305,7 +308,7 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     fence_proxy_async_smem();
     wg_sync(is_dk ? 1 : 2);
     if (r == 0 && ok) {
-      for (int s = 0; s < NSLAB; ++s) tma_store_3d(is_dk ? &tmdK : &tmdV, sOut + s * SLAB_KV, s * 64, rbase + k0, bhk);
+      for (int s = 0; s < NSLAB; ++s) tma_store_4d(is_dk ? &tmdK : &tmdV, sOut + s * SLAB_KV, s * 64, rbase + k0, hk, bt);
       tma_commit_group();
       tma_wait_group<0>();
     }
@@ -321,8 +324,8 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         prefetch_tmap(&tmQ); prefetch_tmap(&tmdO); prefetch_tmap(&tmK); prefetch_tmap(&tmV);
         mbar_expect_tx(bar_kv, 2 * SM::kKV);
         for (int s = 0; s < NSLAB; ++s) {
-          tma_load_3d(sK + s * SLAB_KV, &tmK, bar_kv, s * 64, rbase + k0, bhk);
-          tma_load_3d(sV + s * SLAB_KV, &tmV, bar_kv, s * 64, rbase + k0, bhk);
+          tma_load_4d(sK + s * SLAB_KV, &tmK, bar_kv, s * 64, rbase + k0, hk, bt);
+          tma_load_4d(sV + s * SLAB_KV, &tmV, bar_kv, s * 64, rbase + k0, hk, bt);
         }
         int st = 0, g = 0, t_in = 0;   // stage, head of the group, position in I_h(j): kept incrementally
         uint32_t ph_e = 0;             // parity of the "stage empty" wait (the first NST steps need none)
@@ -335,8 +338,8 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           uint8_t* sdO = sQ + SM::kQS;
           mbar_expect_tx(bar_ld_full + st, SM::kStage + 512);
           for (int s = 0; s < NSLAB; ++s) {
-            tma_load_3d(sQ + s * SLAB_QS, &tmQ, bar_ld_full + st, s * 64, rbase + q0, bhq);
-            tma_load_3d(sdO + s * SLAB_QS, &tmdO, bar_ld_full + st, s * 64, rbase + q0, bhq);
+            tma_load_4d(sQ + s * SLAB_QS, &tmQ, bar_ld_full + st, s * 64, rbase + q0, hq0 + g, bt);
+            tma_load_4d(sdO + s * SLAB_QS, &tmdO, bar_ld_full + st, s * 64, rbase + q0, hq0 + g, bt);
           }
           bulk_load_1d(sVec + st * 128, a.lse2 + (size_t)bhq * vec_stride + pbase + q0, 256, bar_ld_full + st);
           bulk_load_1d(sVec + st * 128 + 64, a.delta + (size_t)bhq * vec_stride + pbase + q0, 256, bar_ld_full + st);
@@ -377,7 +380,7 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           if (lead) {
 #pragma unroll
             for (int kk = 0; kk < BQS / 16; ++kk)
-              mma_ts(tb + d_col, tb + a_col + kk * 8, dB + ((kk * 2048) >> 4), ID_ACC, kk > 0 ? 1u : acc_first);
+              mma_ts(tb + d_col, tb + a_col + (kk >> 1) * 32 + (kk & 1) * 8, dB + ((kk * 2048) >> 4), ID_ACC, kk > 0 ? 1u : acc_first);
           }
         };
         auto gemm_dq = [&](uint32_t d_col, uint64_t dB) {  // dQ^T[D x 64] = K^T dS^T
@@ -434,7 +437,7 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           ok = mbar_wait(bar_ds_ready + b_, par, a.status);
           if (!ok) return;
           tc_fence_after();
-          gemm_acc(cDK, sbuf + 32, dQ_mn0 + st * kStage16, n > 0 ? 1u : 0u);  // dK += dS^T Q
+          gemm_acc(cDK, sbuf + 16, dQ_mn0 + st * kStage16, n > 0 ? 1u : 0u);  // dK += dS^T Q
           commit(bar_ld_empty + st);
           gemm_dq(dpbuf, dDS0 + b_ * kDS16);                                // dQ^T = K^T dS^T over the consumed dP^T(n)
           commit(bar_dq_full + b_);
@@ -460,95 +463,93 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   } else if (warp < 12) {
     setmaxnreg_inc<176>();
     {
-      // ======== two compute warpgroups alternate steps: P^T and dS^T, one KV row per thread ========
-      const int wg = (warp - 4) >> 2;        // steps n with n & 1 == wg, TMEM buffer wg
+      // ======== two compute warpgroups, each takes 32 of the 64 query columns of every step: P^T and dS^T, one
+      // KV row per thread.  Inside the 64-column S^T buffer a warpgroup only ever writes into the 32 columns
+      // it reads: P^T (bf16 pairs) into the first 16 of them, dS^T into the last 16.
+      const int wg = (warp - 4) >> 2;        // query columns [32 wg, 32 wg + 32) of every step
       const int r = (warp & 3) * 32 + lane;  // KV row = TMEM lane
       const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
-      const uint32_t sbuf = t_lane + cS0 + wg * 64, dpbuf = t_lane + cDP0 + wg * 64;
       const int kcol = k0 + r;               // key index of this thread
       const long long kpos = (long long)kcol - off;  // first causal query of this key
       const float2 sc2 = make_float2(a.scale_log2, a.scale_log2);
-      uint8_t* ds_row = sDS + wg * SM::kDS + r * 128;
-      int st = wg % NST, t_in = cnt > 0 ? wg % cnt : 0;   // stage and position in I_h(j) of this warpgroup's next step
-      uint32_t ph_l = (wg / NST) & 1, par = 0;
-      for (int n = wg; n < N && ok; n += 2) {
+      int st = 0, t_in = 0;                  // stage and position in I_h(j) of the next step
+      uint32_t ph_l = 0, par = 0;
+      for (int n = 0; n < N && ok; ++n) {
+        const int b_ = n & 1;
+        const uint32_t sbuf = t_lane + cS0 + b_ * 64 + wg * 32, dpbuf = t_lane + cDP0 + b_ * 64 + wg * 32;
+        uint8_t* ds_row = sDS + b_ * SM::kDS + r * 128;
         const int i = cowa_bwd_tile_at(rg, t_in);
         const int q0 = i * BQS;
         const bool full = cowa_tile_full(w, q0, BQS, k0, BKV, off, Nq, Nk);
-        uint32_t mk[2] = {0xFFFFFFFFu, 0xFFFFFFFFu};
+        uint32_t mk = 0xFFFFFFFFu;
         if (!full) {
           const long long qend = Nq - 1;
-#pragma unroll
-          for (int c = 0; c < 2; ++c) {
-            const long long base = q0 + c * 32;
-            uint32_t m = interval_bits32(kpos, min(kpos + w.n - 1, qend), base);
-            if (w.l > 0)
-              m |= interval_bits32(kpos + w.n + w.g, min(kpos + (long long)w.n + w.g + w.l - 1, qend), base);
-            if (kcol < w.s) m |= interval_bits32(kpos, qend, base);
-            mk[c] = kcol < Nk ? m : 0u;
-          }
+          const long long base = q0 + wg * 32;
+          uint32_t m = interval_bits32(kpos, min(kpos + w.n - 1, qend), base);
+          if (w.l > 0)
+            m |= interval_bits32(kpos + w.n + w.g, min(kpos + (long long)w.n + w.g + w.l - 1, qend), base);
+          if (kcol < w.s) m |= interval_bits32(kpos, qend, base);
+          mk = kcol < Nk ? m : 0u;
         }
-        const float* lse2 = sVec + st * 128;
+        const float* lse2 = sVec + st * 128 + wg * 32;
         const float* dlt = lse2 + 64;
         ok = mbar_wait(bar_ld_full + st, ph_l, a.status);
-        ok = ok && mbar_wait(bar_s_full + wg, par, a.status);
+        ok = ok && mbar_wait(bar_s_full + b_, par, a.status);
         if (!ok) break;
         tc_fence_after();
-        float p[64];
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
+        float p[32];
+        {
           uint32_t sr[32], pk[16];
-          tmem_ld32(sbuf + c * 32, sr);
+          tmem_ld32(sbuf, sr);
           tmem_wait_ld();
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
             const float2 x = fma2(make_float2(__uint_as_float(sr[e]), __uint_as_float(sr[e + 1])), sc2,
-                                  make_float2(-lse2[c * 32 + e], -lse2[c * 32 + e + 1]));
-            p[c * 32 + e] = ex2(x.x);
-            p[c * 32 + e + 1] = ex2(x.y);
+                                  make_float2(-lse2[e], -lse2[e + 1]));
+            p[e] = ex2(x.x);
+            p[e + 1] = ex2(x.y);
           }
           if (!full) {
 #pragma unroll
             for (int e = 0; e < 32; ++e)
-              if (!((mk[c] >> e) & 1u)) p[c * 32 + e] = 0.f;
+              if (!((mk >> e) & 1u)) p[e] = 0.f;
           }
 #pragma unroll
-          for (int e = 0; e < 32; e += 2) pk[e / 2] = pack_bf16(p[c * 32 + e], p[c * 32 + e + 1]);
-          tmem_st16(sbuf + c * 16, pk);  // P^T: 64 queries packed into columns 0-31 of this S^T buffer
+          for (int e = 0; e < 32; e += 2) pk[e / 2] = pack_bf16(p[e], p[e + 1]);
+          tmem_st16(sbuf, pk);  // P^T: this warpgroup's 32 queries as 16 bf16 pairs
         }
         tmem_wait_st();
         tc_fence_before();
-        mbar_arrive(bar_p_ready + wg);
+        mbar_arrive(bar_p_ready + b_);
 
-        ok = mbar_wait(bar_dp_full + wg, par, a.status);
+        ok = mbar_wait(bar_dp_full + b_, par, a.status);
         if (!ok) break;
         tc_fence_after();
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
+        {
           uint32_t dr[32], dsp[16];
-          tmem_ld32(dpbuf + c * 32, dr);
+          tmem_ld32(dpbuf, dr);
           tmem_wait_ld();
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
             const float2 y = add2(make_float2(__uint_as_float(dr[e]), __uint_as_float(dr[e + 1])),
-                                  make_float2(-dlt[c * 32 + e], -dlt[c * 32 + e + 1]));
-            const float2 z = mul2(make_float2(p[c * 32 + e], p[c * 32 + e + 1]), y);
+                                  make_float2(-dlt[e], -dlt[e + 1]));
+            const float2 z = mul2(make_float2(p[e], p[e + 1]), y);
             dsp[e / 2] = pack_bf16(z.x, z.y);
           }
-          tmem_st16(sbuf + 32 + c * 16, dsp);  // dS^T beside P^T, in columns 32-63 of the S^T buffer
+          tmem_st16(sbuf + 16, dsp);  // dS^T beside P^T
           // dS^T also to shared memory (row r = 128 B = 8 chunks, 128B swizzle) for the dQ^T product
 #pragma unroll
           for (int ch = 0; ch < 4; ++ch)
-            *reinterpret_cast<uint4*>(ds_row + (((c * 4 + ch) ^ (r & 7)) << 4)) =
+            *reinterpret_cast<uint4*>(ds_row + (((wg * 4 + ch) ^ (r & 7)) << 4)) =
                 make_uint4(dsp[ch * 4], dsp[ch * 4 + 1], dsp[ch * 4 + 2], dsp[ch * 4 + 3]);
         }
         tmem_wait_st();
         tc_fence_before();
         fence_proxy_async_smem();
-        mbar_arrive(bar_ds_ready + wg);
-        par ^= 1;
-        st += 2; if (st >= NST) { st -= NST; ph_l ^= 1; }
-        t_in += 2; if (t_in >= cnt) t_in -= cnt; if (t_in >= cnt) t_in %= cnt;
+        mbar_arrive(bar_ds_ready + b_);
+        if (b_) par ^= 1;
+        if (++st == NST) { st = 0; ph_l ^= 1; }
+        if (++t_in == cnt) t_in = 0;
       }
       if (wg == 0) store_grad(true);
     }
@@ -581,9 +582,14 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           if (d < D) {
             if (a.dq_fixed) {
               const float fx = a.scale * kDqFixedOne;
+              bool out_of_range = false;
 #pragma unroll
-              for (int c = 0; c < 32; ++c)
-                reinterpret_cast<int*>(stage)[c * D + d] = __float2int_rn(__uint_as_float(v[hf][c]) * fx);
+              for (int c = 0; c < 32; ++c) {
+                const float x = __uint_as_float(v[hf][c]) * fx;
+                out_of_range |= !(fabsf(x) < 2147483520.f);  // the conversion would saturate (or x is not a number)
+                reinterpret_cast<int*>(stage)[c * D + d] = __float2int_rn(x);
+              }
+              if (out_of_range) atomicOr(a.status, (unsigned)COWA_DEV_DQ_RANGE);
             } else {
 #pragma unroll
               for (int c = 0; c < 32; ++c) stage[c * D + d] = __uint_as_float(v[hf][c]) * a.scale;
@@ -592,7 +598,7 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           fence_proxy_async_smem();
           wg_sync(3);
           if (issuer) {
-            tma_reduce_add_3d(&tmdQ, stage, 0, pbase + q0 + hf * 32, bhq);
+            tma_reduce_add_4d(&tmdQ, stage, 0, pbase + q0 + hf * 32, bhq, 0);
             tma_commit_group();
           }
         }
@@ -614,7 +620,8 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 template <int D>
 __global__ void cowa_bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ d_o,
                                            const float* __restrict__ lse, float* __restrict__ lse2,
-                                           float* __restrict__ delta, int T, int Tpad, long long BH) {
+                                           float* __restrict__ delta, int T, int Tpad, long long BH, int H,
+                                           CowaStrides so) {
   constexpr int TPR = D / 8;  // threads per row (16 bytes each)
   const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const long long row = gid / TPR;
@@ -624,7 +631,7 @@ __global__ void cowa_bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, 
   const int t = (int)(row % Tpad);
   float s = 0.f;
   if (t < T) {
-    const size_t base = ((size_t)bh * T + t) * D + part * 8;
+    const size_t base = (size_t)(bh / H) * so.b + (size_t)(bh % H) * so.h + (size_t)t * so.t + part * 8;
     const uint4 x = *reinterpret_cast<const uint4*>(o + base);
     const uint4 y = *reinterpret_cast<const uint4*>(d_o + base);
     const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
@@ -644,7 +651,8 @@ __global__ void cowa_bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, 
 
 template <int D>
 __global__ void cowa_bwd_convert_dq_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dq, int T,
-                                           int Tpad, long long BH, int fixed) {
+                                           int Tpad, long long BH, int fixed, int H, CowaStrides sq,
+                                           unsigned int* status) {
   const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;  // one thread per 8 elements
   const long long total = BH * T * (D / 8);
   if (gid >= total) return;
@@ -658,10 +666,14 @@ __global__ void cowa_bwd_convert_dq_kernel(const float* __restrict__ acc, __nv_b
     const float u = 1.f / kDqFixedOne;
     x = make_float4(__float_as_int(x.x) * u, __float_as_int(x.y) * u, __float_as_int(x.z) * u, __float_as_int(x.w) * u);
     y = make_float4(__float_as_int(y.x) * u, __float_as_int(y.y) * u, __float_as_int(y.z) * u, __float_as_int(y.w) * u);
+    // half of the representable range: a total that wrapped around lands out here in most cases
+    const float big = fmaxf(fmaxf(fmaxf(fabsf(x.x), fabsf(x.y)), fmaxf(fabsf(x.z), fabsf(x.w))),
+                            fmaxf(fmaxf(fabsf(y.x), fabsf(y.y)), fmaxf(fabsf(y.z), fabsf(y.w))));
+    if (big >= 4096.f) atomicOr(status, (unsigned)COWA_DEV_DQ_RANGE);
   }
   uint4 v;
   v.x = pack_bf16(x.x, x.y); v.y = pack_bf16(x.z, x.w); v.z = pack_bf16(y.x, y.y); v.w = pack_bf16(y.z, y.w);
-  *reinterpret_cast<uint4*>(dq + ((size_t)bh * T + t) * D + part * 8) = v;
+  *reinterpret_cast<uint4*>(dq + (size_t)(bh / H) * sq.b + (size_t)(bh % H) * sq.h + (size_t)t * sq.t + part * 8) = v;
 }
 
 // Packed batches.  One block per (64-row chunk of the padded row space, QO head): Delta and LSE * log2(e)
@@ -704,7 +716,8 @@ __global__ void cowa_bwd_preprocess_varlen_kernel(const __nv_bfloat16* __restric
 // Packed batches: fp32 (or fixed-point) dQ accumulator in the padded row space -> bf16 dq in the packed one.
 template <int D>
 __global__ void cowa_bwd_convert_dq_varlen_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dq,
-                                                  const int* __restrict__ cu, int B, int total, int Tpad, int fixed) {
+                                                  const int* __restrict__ cu, int B, int total, int Tpad, int fixed,
+                                                  unsigned int* status) {
   constexpr int TPR = D / 8;
   const int chunk = blockIdx.x, h = blockIdx.y;
   const int r = threadIdx.x / TPR, part = threadIdx.x % TPR;
@@ -719,6 +732,9 @@ __global__ void cowa_bwd_convert_dq_varlen_kernel(const float* __restrict__ acc,
     const float u = 1.f / kDqFixedOne;
     x = make_float4(__float_as_int(x.x) * u, __float_as_int(x.y) * u, __float_as_int(x.z) * u, __float_as_int(x.w) * u);
     y = make_float4(__float_as_int(y.x) * u, __float_as_int(y.y) * u, __float_as_int(y.z) * u, __float_as_int(y.w) * u);
+    const float big = fmaxf(fmaxf(fmaxf(fabsf(x.x), fabsf(x.y)), fmaxf(fabsf(x.z), fabsf(x.w))),
+                            fmaxf(fmaxf(fabsf(y.x), fabsf(y.y)), fmaxf(fabsf(y.z), fabsf(y.w))));
+    if (big >= 4096.f) atomicOr(status, (unsigned)COWA_DEV_DQ_RANGE);
   }
   uint4 v;
   v.x = pack_bf16(x.x, x.y); v.y = pack_bf16(x.z, x.w); v.z = pack_bf16(y.x, y.y); v.w = pack_bf16(y.z, y.w);
@@ -728,7 +744,8 @@ __global__ void cowa_bwd_convert_dq_varlen_kernel(const float* __restrict__ acc,
 // Sum of the per-block partial dK, dV (heads of a group spread over `parts` blocks), in slot order, to bf16.
 template <int D>
 __global__ void cowa_bwd_reduce_dkv_kernel(const float* __restrict__ part, __nv_bfloat16* __restrict__ dk,
-                                           __nv_bfloat16* __restrict__ dv, int T, int nKV, int parts, long long BHk) {
+                                           __nv_bfloat16* __restrict__ dv, int T, int nKV, int parts, long long BHk,
+                                           int H, CowaStrides sk, CowaStrides sv) {
   const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;  // one thread per 8 elements of dK and dV
   const long long total = BHk * nKV * BKV * (D / 8);
   if (gid >= total) return;
@@ -758,19 +775,31 @@ __global__ void cowa_bwd_reduce_dkv_kernel(const float* __restrict__ part, __nv_
     uint4 v;
     v.x = pack_bf16(acc[m][0], acc[m][1]); v.y = pack_bf16(acc[m][2], acc[m][3]);
     v.z = pack_bf16(acc[m][4], acc[m][5]); v.w = pack_bf16(acc[m][6], acc[m][7]);
-    *reinterpret_cast<uint4*>((m == 0 ? dk : dv) + ((size_t)bhk * T + t) * D + ch * 8) = v;
+    const CowaStrides& sg = m == 0 ? sk : sv;
+    *reinterpret_cast<uint4*>((m == 0 ? dk : dv) + (size_t)(bhk / H) * sg.b + (size_t)(bhk % H) * sg.h + (size_t)t * sg.t + ch * 8) = v;
   }
 }
-
-// Optional CUDA events recorded around the main kernel of the next cowa_bwd calls on this host thread.
-thread_local cudaEvent_t g_ev_main_start = nullptr, g_ev_main_stop = nullptr;
 
 // Blocks per KV tile.  A block normally takes the whole GQA group of its KV tile (dK, dV then never leave
 // TMEM).  That starves the GPU when B * Hkv * tiles is small, and it makes the sink tiles -- visited by
 // every query tile of every head -- the critical path when Hkv is small; in both cases the group's heads
 // are spread over `parts` blocks (a divisor of G), chosen as the smallest that gives two waves of
 // blocks and keeps the longest block under 3/4 of an even share of the work.
-constexpr int kSMs = 148;
+int sm_count() {
+  static int cached = 0;
+  if (cached == 0) {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&
+        n > 0)
+      cached = n;
+    else {
+      cudaGetLastError();
+      return 148;  // B200; used when no device can be queried (workspace sizing on a machine without a GPU)
+    }
+  }
+  return cached;
+}
+
 int bwd_parts(int B, int Nq, int Nk, int Hkv, int G, const CowaHeadWindows& hw) {
   const int nKV = (Nk + BKV - 1) / BKV;
   long long total = 0, longest = 0;
@@ -786,6 +815,7 @@ int bwd_parts(int B, int Nq, int Nk, int Hkv, int G, const CowaHeadWindows& hw) 
   total *= (long long)B * G;
   longest *= G;
   const long long blocks = (long long)B * Hkv * nKV;
+  const int kSMs = sm_count();
   for (int p = 1; p < G; ++p) {
     if (G % p) continue;
     if (blocks * p >= 2 * kSMs && longest * 4 * kSMs <= 3 * total * p) return p;
@@ -803,6 +833,13 @@ size_t ws_bytes(int B, int Nq, int Nk, int Hq, int Hkv, int D, int parts) {
   return (size_t)B * Hq * Tpad * ((size_t)D + 2) * sizeof(float) + part_bytes(B, Nk, Hkv, D, parts);
 }
 
+// Contiguous [H, T, D] (x batch) strides.
+CowaStrides packed_strides(int H, long long T, int D) {
+  CowaStrides st;
+  st.t = D; st.h = T * D; st.b = (long long)H * T * D;
+  return st;
+}
+
 template <int D>
 int launch_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* d_o,
                void* dq, void* dk, void* dv, int B, int Nq, int Nk, int Hq, int Hkv, const cowa_params_t* p,
@@ -814,24 +851,24 @@ int launch_bwd(const void* q, const void* k, const void* v, const void* o, const
   float* lse2 = dq_acc + (size_t)BH * Tpad * D;
   float* delta = lse2 + (size_t)BH * Tpad;
   float* dkv_part = delta + (size_t)BH * Tpad;
-  COWA_CUDA_TRY(cudaMemsetAsync(dq_acc, 0, (size_t)BH * Tpad * D * sizeof(float), st));
-  {
-    const long long threads = BH * Tpad * (D / 8);
-    cowa_bwd_preprocess_kernel<D><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(
-        static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse, lse2, delta, T, Tpad, BH);
-    COWA_CUDA_TRY(cudaGetLastError());
-  }
-  CUtensorMap mq, mk, mv, mdo, mdk, mdv, mdq;
+  // Everything that can fail is done before the first launch: strides, tensor maps, the status word.
   int rc;
-  if ((rc = cowa::make_tensor_map_3d(&mdq, dq_acc, p->deterministic ? cowa::MapType::S32 : cowa::MapType::F32, D, Tpad, BH, D,
-                                     32, false)))
+  CowaStrides sq, sk, sv, so;
+  if ((rc = cowa::resolve_strides(p->q_strides, Hq, Nq, D, &sq))) return rc;
+  if ((rc = cowa::resolve_strides(p->k_strides, Hkv, Nk, D, &sk))) return rc;
+  if ((rc = cowa::resolve_strides(p->v_strides, Hkv, Nk, D, &sv))) return rc;
+  if ((rc = cowa::resolve_strides(p->o_strides, Hq, Nq, D, &so))) return rc;
+  if (BH > 0x7FFFFFFFll) return COWA_ERR_UNSUPPORTED;
+  CUtensorMap mq, mk, mv, mdo, mdk, mdv, mdq;
+  if ((rc = cowa::make_tensor_map(&mdq, dq_acc, p->deterministic ? cowa::MapType::S32 : cowa::MapType::F32, D, Tpad, (int)BH,
+                                  1, packed_strides((int)BH, Tpad, D), D, 32, false)))
     return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mq, q, cowa::MapType::BF16, D, T, BH, 64, BQS))) return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mdo, d_o, cowa::MapType::BF16, D, T, BH, 64, BQS))) return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mk, k, cowa::MapType::BF16, D, Nk, (long long)B * Hkv, 64, BKV))) return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mv, v, cowa::MapType::BF16, D, Nk, (long long)B * Hkv, 64, BKV))) return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mdk, dk, cowa::MapType::BF16, D, Nk, (long long)B * Hkv, 64, BKV))) return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mdv, dv, cowa::MapType::BF16, D, Nk, (long long)B * Hkv, 64, BKV))) return rc;
+  if ((rc = cowa::make_tensor_map(&mq, q, cowa::MapType::BF16, D, T, Hq, B, sq, 64, BQS))) return rc;
+  if ((rc = cowa::make_tensor_map(&mdo, d_o, cowa::MapType::BF16, D, T, Hq, B, so, 64, BQS))) return rc;
+  if ((rc = cowa::make_tensor_map(&mk, k, cowa::MapType::BF16, D, Nk, Hkv, B, sk, 64, BKV))) return rc;
+  if ((rc = cowa::make_tensor_map(&mv, v, cowa::MapType::BF16, D, Nk, Hkv, B, sv, 64, BKV))) return rc;
+  if ((rc = cowa::make_tensor_map(&mdk, dk, cowa::MapType::BF16, D, Nk, Hkv, B, sk, 64, BKV))) return rc;
+  if ((rc = cowa::make_tensor_map(&mdv, dv, cowa::MapType::BF16, D, Nk, Hkv, B, sv, 64, BKV))) return rc;
   BwdArgs a;
   a.lse2 = lse2; a.delta = delta; a.dq_acc = dq_acc;
   a.status = cowa::device_status_word();
@@ -846,28 +883,36 @@ int launch_bwd(const void* q, const void* k, const void* v, const void* o, const
   a.cu = nullptr; a.dk = nullptr; a.dv = nullptr; a.total = 0; a.tiles_bound = 0;
   a.sink = 0; a.local = 0; a.hkv_global = 0; a.hkv_offset = 0; a.full_attn = 0; a.explicit_windows = 0;
   for (int h = 0; h < Hkv; ++h) {
-    const int sk = hw.w[h].s < Nk ? hw.w[h].s : Nk;
-    a.sink_tiles = std::max(a.sink_tiles, (sk + BKV - 1) / BKV);
+    const int sk_ = hw.w[h].s < Nk ? hw.w[h].s : Nk;
+    a.sink_tiles = std::max(a.sink_tiles, (sk_ + BKV - 1) / BKV);
   }
-  COWA_CUDA_TRY(cudaFuncSetAttribute(cowa_bwd_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     BwdSmem<D>::kBytes));
   const long long nblocks = (long long)((Nk + BKV - 1) / BKV) * B * Hkv * parts;
   if (nblocks > 0x7FFFFFFFll) return COWA_ERR_UNSUPPORTED;
-  if (g_ev_main_start) COWA_CUDA_TRY(cudaEventRecord(g_ev_main_start, st));
+  COWA_CUDA_TRY(cudaFuncSetAttribute(cowa_bwd_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     BwdSmem<D>::kBytes));
+  COWA_CUDA_TRY(cudaMemsetAsync(dq_acc, 0, (size_t)BH * Tpad * D * sizeof(float), st));
+  {
+    const long long threads = BH * Tpad * (D / 8);
+    cowa_bwd_preprocess_kernel<D><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(
+        static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse, lse2, delta, T, Tpad, BH, Hq, so);
+    COWA_CUDA_TRY(cudaGetLastError());
+  }
+  if (p->bwd_main_start_event) COWA_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(p->bwd_main_start_event), st));
   cowa_bwd_kernel<D, false><<<(unsigned)nblocks, 512, BwdSmem<D>::kBytes, st>>>(mq, mk, mv, mdo, mdk, mdv, mdq, a);
   COWA_CUDA_TRY(cudaGetLastError());
-  if (g_ev_main_stop) COWA_CUDA_TRY(cudaEventRecord(g_ev_main_stop, st));
+  if (p->bwd_main_stop_event) COWA_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(p->bwd_main_stop_event), st));
   {
     const long long threads = BH * T * (D / 8);
     cowa_bwd_convert_dq_kernel<D><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(
-        dq_acc, static_cast<__nv_bfloat16*>(dq), T, Tpad, BH, p->deterministic ? 1 : 0);
+        dq_acc, static_cast<__nv_bfloat16*>(dq), T, Tpad, BH, p->deterministic ? 1 : 0, Hq, sq, a.status);
     COWA_CUDA_TRY(cudaGetLastError());
   }
   if (parts > 1) {
     const int nKV = (Nk + BKV - 1) / BKV;
     const long long threads = (long long)B * Hkv * nKV * BKV * (D / 8);
     cowa_bwd_reduce_dkv_kernel<D><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(
-        dkv_part, static_cast<__nv_bfloat16*>(dk), static_cast<__nv_bfloat16*>(dv), Nk, nKV, parts, (long long)B * Hkv);
+        dkv_part, static_cast<__nv_bfloat16*>(dk), static_cast<__nv_bfloat16*>(dv), Nk, nKV, parts, (long long)B * Hkv,
+        Hkv, sk, sv);
     COWA_CUDA_TRY(cudaGetLastError());
   }
   return COWA_OK;
@@ -888,22 +933,19 @@ int launch_bwd_varlen(const void* q, const void* k, const void* v, const void* o
   float* dq_acc = static_cast<float*>(ws);
   float* lse2 = dq_acc + (size_t)Hq * Tpad * D;
   float* delta = lse2 + (size_t)Hq * Tpad;
-  COWA_CUDA_TRY(cudaMemsetAsync(dq_acc, 0, (size_t)Hq * Tpad * D * sizeof(float), st));
-  const dim3 chunks(Tpad / BQS, Hq);
-  cowa_bwd_preprocess_varlen_kernel<D><<<chunks, BQS * (D / 8), 0, st>>>(
-      static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse, lse2, delta, cu, B, total, Tpad);
-  COWA_CUDA_TRY(cudaGetLastError());
+  if (cowa::any_stride_set(p)) return COWA_ERR_UNSUPPORTED;  // packed tensors are contiguous [H, total, D]
   CUtensorMap mq, mk, mv, mdo, mdk, mdv, mdq;
   int rc;
-  if ((rc = cowa::make_tensor_map_3d(&mdq, dq_acc, p->deterministic ? cowa::MapType::S32 : cowa::MapType::F32, D, Tpad, Hq, D,
-                                     32, false)))
+  const CowaStrides sq = packed_strides(Hq, total, D), sk = packed_strides(Hkv, total, D);
+  if ((rc = cowa::make_tensor_map(&mdq, dq_acc, p->deterministic ? cowa::MapType::S32 : cowa::MapType::F32, D, Tpad, Hq, 1,
+                                  packed_strides(Hq, Tpad, D), D, 32, false)))
     return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mq, q, cowa::MapType::BF16, D, total, Hq, 64, BQS))) return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mdo, d_o, cowa::MapType::BF16, D, total, Hq, 64, BQS))) return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mk, k, cowa::MapType::BF16, D, total, Hkv, 64, BKV))) return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mv, v, cowa::MapType::BF16, D, total, Hkv, 64, BKV))) return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mdk, dk, cowa::MapType::BF16, D, total, Hkv, 64, BKV))) return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mdv, dv, cowa::MapType::BF16, D, total, Hkv, 64, BKV))) return rc;
+  if ((rc = cowa::make_tensor_map(&mq, q, cowa::MapType::BF16, D, total, Hq, 1, sq, 64, BQS))) return rc;
+  if ((rc = cowa::make_tensor_map(&mdo, d_o, cowa::MapType::BF16, D, total, Hq, 1, sq, 64, BQS))) return rc;
+  if ((rc = cowa::make_tensor_map(&mk, k, cowa::MapType::BF16, D, total, Hkv, 1, sk, 64, BKV))) return rc;
+  if ((rc = cowa::make_tensor_map(&mv, v, cowa::MapType::BF16, D, total, Hkv, 1, sk, 64, BKV))) return rc;
+  if ((rc = cowa::make_tensor_map(&mdk, dk, cowa::MapType::BF16, D, total, Hkv, 1, sk, 64, BKV))) return rc;
+  if ((rc = cowa::make_tensor_map(&mdv, dv, cowa::MapType::BF16, D, total, Hkv, 1, sk, 64, BKV))) return rc;
   BwdArgs a;
   a.lse2 = lse2; a.delta = delta; a.dq_acc = dq_acc;
   a.status = cowa::device_status_word();
@@ -915,8 +957,8 @@ int launch_bwd_varlen(const void* q, const void* k, const void* v, const void* o
   a.sink_tiles = 0;  // KV tiles per sequence that hold sink columns (launched first)
   if (!p->full_attn)
     for (int h = 0; h < Hkv; ++h) {
-      const int sk = std::min(p->windows ? hw.w[h].s : p->sink, total);
-      a.sink_tiles = std::max(a.sink_tiles, (sk + BKV - 1) / BKV);
+      const int sk_ = std::min(p->windows ? hw.w[h].s : p->sink, total);
+      a.sink_tiles = std::max(a.sink_tiles, (sk_ + BKV - 1) / BKV);
     }
   a.dq_fixed = p->deterministic ? 1 : 0;
   a.parts = 1; a.dkv_part = nullptr;
@@ -925,16 +967,21 @@ int launch_bwd_varlen(const void* q, const void* k, const void* v, const void* o
   a.sink = p->sink; a.local = p->local;
   a.hkv_global = p->hkv_global > 0 ? p->hkv_global : Hkv;
   a.hkv_offset = p->hkv_offset; a.full_attn = p->full_attn; a.explicit_windows = p->windows != nullptr;
-  COWA_CUDA_TRY(cudaFuncSetAttribute(cowa_bwd_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     BwdSmem<D>::kBytes));
   const long long nblocks = (long long)a.tiles_bound * Hkv + (long long)a.sink_tiles * B * Hkv;
   if (nblocks > 0x7FFFFFFFll) return COWA_ERR_UNSUPPORTED;
-  if (g_ev_main_start) COWA_CUDA_TRY(cudaEventRecord(g_ev_main_start, st));
+  COWA_CUDA_TRY(cudaFuncSetAttribute(cowa_bwd_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     BwdSmem<D>::kBytes));
+  COWA_CUDA_TRY(cudaMemsetAsync(dq_acc, 0, (size_t)Hq * Tpad * D * sizeof(float), st));
+  const dim3 chunks(Tpad / BQS, Hq);
+  cowa_bwd_preprocess_varlen_kernel<D><<<chunks, BQS * (D / 8), 0, st>>>(
+      static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse, lse2, delta, cu, B, total, Tpad);
+  COWA_CUDA_TRY(cudaGetLastError());
+  if (p->bwd_main_start_event) COWA_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(p->bwd_main_start_event), st));
   cowa_bwd_kernel<D, true><<<(unsigned)nblocks, 512, BwdSmem<D>::kBytes, st>>>(mq, mk, mv, mdo, mdk, mdv, mdq, a);
   COWA_CUDA_TRY(cudaGetLastError());
-  if (g_ev_main_stop) COWA_CUDA_TRY(cudaEventRecord(g_ev_main_stop, st));
+  if (p->bwd_main_stop_event) COWA_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(p->bwd_main_stop_event), st));
   cowa_bwd_convert_dq_varlen_kernel<D><<<chunks, BQS * (D / 8), 0, st>>>(dq_acc, static_cast<__nv_bfloat16*>(dq), cu, B,
-                                                                        total, Tpad, p->deterministic ? 1 : 0);
+                                                                        total, Tpad, p->deterministic ? 1 : 0, a.status);
   COWA_CUDA_TRY(cudaGetLastError());
   return COWA_OK;
 }
@@ -969,12 +1016,6 @@ int cowa_bwd_varlen(const void* q, const void* k, const void* v, const void* o, 
                                            workspace, st)
                   : launch_bwd_varlen<64>(q, k, v, o, lse, d_o, dq, dk, dv, cu_seqlens, B, total, Hq, Hkv, p, hw,
                                           workspace, st);
-}
-
-int cowa_bwd_set_profile_events(void* start_event, void* stop_event) {
-  g_ev_main_start = static_cast<cudaEvent_t>(start_event);
-  g_ev_main_stop = static_cast<cudaEvent_t>(stop_event);
-  return COWA_OK;
 }
 
 size_t cowa_bwd_prefill_workspace_bytes(int B, int Nq, int Nk, int Hq, int Hkv, int D, const cowa_params_t* p) {

@@ -58,6 +58,7 @@ struct DecodeArgs {
   float* ws_m;  // [B, Hq, S]
   float* ws_l;  // [B, Hq, S]
   int B, Tmax, Hq, Hkv, S;
+  CowaStrides sk, sv;  // element strides (batch, head, token) of the contiguous-row cache
   int sink, near, hkv_global, hkv_offset, full_attn;
   float scale_log2;
   // extended kernel only: several newest tokens per sequence and / or a paged cache
@@ -131,7 +132,7 @@ __global__ void __launch_bounds__(kThreads, 5) cowa_decode_split_kernel(const De
   };
   auto col_valid = [&](int c) -> bool { return EXT ? (c < G && tq0 + c / gsz <= tq1) : (c < G); };
   // address of cache row `tok` of this (sequence, KV head)
-  auto row_ptr = [&](const __nv_bfloat16* base, int tok) -> const __nv_bfloat16* {
+  auto row_ptr = [&](const __nv_bfloat16* base, const CowaStrides& cs, int tok) -> const __nv_bfloat16* {
     if constexpr (EXT) {
       if (a.block_table) {
         // page sizes are almost always powers of two: shift and mask instead of a runtime division
@@ -141,7 +142,7 @@ __global__ void __launch_bounds__(kThreads, 5) cowa_decode_split_kernel(const De
         return base + (((size_t)pg * a.Hkv + hk) * a.page_size + po) * D;
       }
     }
-    return base + ((size_t)b * a.Hkv + hk) * (size_t)a.Tmax * D + (size_t)tok * D;
+    return base + (size_t)b * cs.b + (size_t)hk * cs.h + (size_t)tok * cs.t;
   };
   VisMap vm;
   vm.lo0 = rg[0].lo; vm.n0 = nr > 0 ? rg[0].hi - rg[0].lo + 1 : 0;
@@ -181,8 +182,8 @@ __global__ void __launch_bounds__(kThreads, 5) cowa_decode_split_kernel(const De
       const int rA = blk * 16 + g, rB = rA + 8;
       const int tokA = vm.token(c0 + min(rA, clen - 1));
       const int tokB = vm.token(c0 + min(rB, clen - 1));
-      const __nv_bfloat16* pa = row_ptr(a.kc, tokA) + t * 8;
-      const __nv_bfloat16* pb = row_ptr(a.kc, tokB) + t * 8;
+      const __nv_bfloat16* pa = row_ptr(a.kc, a.sk, tokA) + t * 8;
+      const __nv_bfloat16* pb = row_ptr(a.kc, a.sk, tokB) + t * 8;
       uint4 ka[KC], kb[KC];
 #pragma unroll
       for (int cc = 0; cc < KC; ++cc) { ka[cc] = ldg128(pa + cc * 32); kb[cc] = ldg128(pb + cc * 32); }
@@ -255,7 +256,7 @@ __global__ void __launch_bounds__(kThreads, 5) cowa_decode_split_kernel(const De
       uint4 vv[4][NB];
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
-        const __nv_bfloat16* src = row_ptr(a.vc, vm.token(c0 + min(rr[k], clen - 1))) + g * 8;
+        const __nv_bfloat16* src = row_ptr(a.vc, a.sv, vm.token(c0 + min(rr[k], clen - 1))) + g * 8;
 #pragma unroll
         for (int bb = 0; bb < NB; ++bb) vv[k][bb] = ldg128(src + bb * 64);
       }
@@ -505,7 +506,10 @@ int decode_validate(const void* q, const void* kc, const void* vc, const int32_t
   const int G = Hq / Hkv;
   if (G != 1 && G != 2 && G != 4 && G != 8) return COWA_ERR_UNSUPPORTED;
   if (B > 65535 || Hkv > 65535) return COWA_ERR_UNSUPPORTED;
+  if (!(p->softmax_scale > 0.f)) return COWA_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(kc) || !aligned16(vc) || !aligned16(o)) return COWA_ERR_MISALIGNED;
+  for (int i = 0; i < 3; ++i)
+    if (p->q_strides[i] || p->o_strides[i]) return COWA_ERR_UNSUPPORTED;  // q and o of a decode step are [B, Hq, D]
   *S = pick_splits(B, Tmax, Hq, Hkv, D, p);
   return COWA_OK;
 }
@@ -527,6 +531,9 @@ int decode_launch(const void* q, const void* kc, const void* vc, const int32_t* 
   a.ws_m = a.ws_o + (size_t)B * Hq * S * D;
   a.ws_l = a.ws_m + (size_t)B * Hq * S;
   a.B = B; a.Tmax = Tmax; a.Hq = Hq; a.Hkv = Hkv; a.S = S;
+  int rc;
+  if ((rc = resolve_strides(p->k_strides, Hkv, Tmax, D, &a.sk))) return rc;
+  if ((rc = resolve_strides(p->v_strides, Hkv, Tmax, D, &a.sv))) return rc;
   a.sink = p->sink; a.near = p->local;
   a.hkv_global = p->hkv_global > 0 ? p->hkv_global : Hkv;
   a.hkv_offset = p->hkv_offset;
@@ -557,6 +564,9 @@ int decode_ext_launch(const void* q, const void* kc, const void* vc, const int32
   a.ws_m = a.ws_o + rows * S * D;
   a.ws_l = a.ws_m + rows * S;
   a.B = B; a.Tmax = Tmax; a.Hq = Hq; a.Hkv = Hkv; a.S = S;
+  const int64_t none[3] = {0, 0, 0};
+  resolve_strides(none, Hkv, Tmax, D, &a.sk);  // contiguous [B, Hkv, Tmax, D] (paged: rows are addressed through the table)
+  a.sv = a.sk;
   a.sink = p->sink; a.near = p->local;
   a.hkv_global = p->hkv_global > 0 ? p->hkv_global : Hkv;
   a.hkv_offset = p->hkv_offset;
@@ -593,6 +603,7 @@ static int decode_ext(const void* q, const void* kc, const void* vc, const int32
   int st = cowa::decode_validate(q, kc, vc, lens, o, B, Tmax, Hq, Hkv, D, p, &S);
   if (st != COWA_OK) return st;
   if (Nq <= 0 || Nq > 64 || !workspace) return COWA_ERR_INVALID_ARG;
+  if (cowa::any_stride_set(p)) return COWA_ERR_UNSUPPORTED;
   if ((long long)B * ((Nq + 7) / 8 * 8) > 65535) return COWA_ERR_UNSUPPORTED;
   if (!cowa::aligned16(workspace)) return COWA_ERR_MISALIGNED;
   S = pick_splits_ext(B, Nq, Tmax, Hq, Hkv, D, p);

@@ -109,15 +109,15 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   // Sequence geometry.  Packed batches: every sequence has its own N_q <= N_k, its rows start at
   // cu_q[b] / cu_k[b] of a [H, total, D] tensor, and its windows follow from its own N_k.
   int Nq = a.Nq, Nk = a.Nk, qbase = 0, kbase = 0;
-  int bhq = b * a.Hq + h, bhk = b * a.Hkv + hk;
+  int bt = b;  // batch coordinate of the tensor maps (packed tensors have none)
   CowaWin w = a.wins.w[hk];
   if constexpr (VARLEN) {
     qbase = a.cu_q[b]; Nq = a.cu_q[b + 1] - qbase;
     kbase = a.cu_k[b]; Nk = a.cu_k[b + 1] - kbase;
-    bhq = h; bhk = hk;
+    bt = 0;
     if (Nq > Nk || qbase < 0 || kbase < 0 || qbase + Nq > a.total_q || kbase + Nk > a.total_k) {
       // malformed offsets: report, touch nothing
-      if (threadIdx.x == 0) atomicOr(a.status, 2u);
+      if (threadIdx.x == 0) atomicOr(a.status, (unsigned)COWA_DEV_BAD_SEQLENS);
       return;
     }
     if (a.full_attn) { w.s = 0; w.n = Nk; w.g = 0; w.l = 0; }
@@ -166,7 +166,7 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           const int j = cowa_fwd_tile_at(rg, t);
           uint8_t* dst = sK + (t & 1) * SM::kKV;
           mbar_expect_tx(bar_k + (t & 1), SM::kKV);
-          for (int s = 0; s < NSLAB; ++s) tma_load_3d(dst + s * SLAB_K, &tmK, bar_k + (t & 1), s * 64, kbase + j * BK, bhk);
+          for (int s = 0; s < NSLAB; ++s) tma_load_4d(dst + s * SLAB_K, &tmK, bar_k + (t & 1), s * 64, kbase + j * BK, hk, bt);
         }
       };
       auto load_v = [&](int t) {
@@ -174,7 +174,7 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           const int j = cowa_fwd_tile_at(rg, t);
           uint8_t* dst = sV + (t & 1) * SM::kKV;
           mbar_expect_tx(bar_v + (t & 1), SM::kKV);
-          for (int s = 0; s < NSLAB; ++s) tma_load_3d(dst + s * SLAB_K, &tmV, bar_v + (t & 1), s * 64, kbase + j * BK, bhk);
+          for (int s = 0; s < NSLAB; ++s) tma_load_4d(dst + s * SLAB_K, &tmV, bar_v + (t & 1), s * 64, kbase + j * BK, hk, bt);
         }
       };
       auto issue_s = [&](int buf) {  // S = Q K^T into TMEM buffer buf from K buffer buf
@@ -190,7 +190,7 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       if (lead) {
         prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV);
         mbar_expect_tx(bar_q, SM::kQ);
-        for (int s = 0; s < NSLAB; ++s) tma_load_3d(sQ + s * SLAB_Q, &tmQ, bar_q, s * 64, qbase + q0, bhq);
+        for (int s = 0; s < NSLAB; ++s) tma_load_4d(sQ + s * SLAB_Q, &tmQ, bar_q, s * 64, qbase + q0, h, bt);
       }
       load_k(0);
       if (nt > 1) load_k(1);
@@ -390,14 +390,14 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         }
       }
       if (row_valid) {
-        const size_t li = VARLEN ? (size_t)h * a.total_q + qbase + row : (size_t)bhq * Nq + row;
+        const size_t li = VARLEN ? (size_t)h * a.total_q + qbase + row : ((size_t)b * a.Hq + h) * Nq + row;
         a.lse[li] = 0.6931471805599453f * (m_ref + log2f(l_sum));
       }
       fence_proxy_async_smem();
     }
     asm volatile("bar.sync 1, 128;" ::: "memory");  // the four softmax warps
     if (tid == 0 && ok && nt > 0 && !tail_rows) {
-      for (int s = 0; s < NSLAB; ++s) tma_store_3d(&tmO, sQ + s * SLAB_Q, s * 64, qbase + q0, bhq);
+      for (int s = 0; s < NSLAB; ++s) tma_store_4d(&tmO, sQ + s * SLAB_Q, s * 64, qbase + q0, h, bt);
       tma_commit_group();
       tma_wait_group<0>();
     }
@@ -421,11 +421,17 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
   CUtensorMap mq, mk, mv, mo;
   int rc;
   const int rows_q = VARLEN ? total_q : Nq, rows_k = VARLEN ? total_k : Nk;
-  const long long nq_maps = VARLEN ? Hq : (long long)B * Hq, nk_maps = VARLEN ? Hkv : (long long)B * Hkv;
-  if ((rc = cowa::make_tensor_map_3d(&mq, q, cowa::MapType::BF16, D, rows_q, nq_maps, 64, BQ))) return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mk, k, cowa::MapType::BF16, D, rows_k, nk_maps, 64, BK))) return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mv, v, cowa::MapType::BF16, D, rows_k, nk_maps, 64, BK))) return rc;
-  if ((rc = cowa::make_tensor_map_3d(&mo, o, cowa::MapType::BF16, D, rows_q, nq_maps, 64, BQ))) return rc;
+  const int nb = VARLEN ? 1 : B;  // packed tensors are [H, total, D]
+  CowaStrides sq, sk, sv, so;
+  if (VARLEN && cowa::any_stride_set(p)) return COWA_ERR_UNSUPPORTED;
+  if ((rc = cowa::resolve_strides(p->q_strides, Hq, rows_q, D, &sq))) return rc;
+  if ((rc = cowa::resolve_strides(p->k_strides, Hkv, rows_k, D, &sk))) return rc;
+  if ((rc = cowa::resolve_strides(p->v_strides, Hkv, rows_k, D, &sv))) return rc;
+  if ((rc = cowa::resolve_strides(p->o_strides, Hq, rows_q, D, &so))) return rc;
+  if ((rc = cowa::make_tensor_map(&mq, q, cowa::MapType::BF16, D, rows_q, Hq, nb, sq, 64, BQ))) return rc;
+  if ((rc = cowa::make_tensor_map(&mk, k, cowa::MapType::BF16, D, rows_k, Hkv, nb, sk, 64, BK))) return rc;
+  if ((rc = cowa::make_tensor_map(&mv, v, cowa::MapType::BF16, D, rows_k, Hkv, nb, sv, 64, BK))) return rc;
+  if ((rc = cowa::make_tensor_map(&mo, o, cowa::MapType::BF16, D, rows_q, Hq, nb, so, 64, BQ))) return rc;
   FwdArgs a;
   a.lse = lse;
   a.status = cowa::device_status_word();

@@ -20,9 +20,18 @@ TOL_MAX, TOL_MEAN, TOL_LSE = 2e-2, 2e-3, 1e-3
 DEV = "cuda"
 
 
+MEASURED = {}  # (configuration, tensor) -> [max-abs error, sum of mean-abs errors, checks]; written out by conftest.py
+_CONFIG = [None]
+
+
 def check(name, got, want, tol_max=TOL_MAX, tol_mean=TOL_MEAN, rtol=0.0, rtol_mean=0.0):
     got = np.asarray(got, dtype=np.float64)
     err = np.abs(got - want)
+    if _CONFIG[0] is not None and np.isfinite(err).all():
+        tensor = name.replace(_CONFIG[0], "").split("[")[0].split()[-1]
+        rec = MEASURED.setdefault((_CONFIG[0], tensor), [0.0, 0.0, 0, 0.0])
+        rec[0] = max(rec[0], float(err.max())); rec[1] += float(err.mean()); rec[2] += 1
+        rec[3] = max(rec[3], float(np.abs(want).max()))
     assert np.isfinite(got).all(), f"{name}: non-finite output"
     excess = err - rtol * np.abs(want)
     assert excess.max() <= tol_max, f"{name}: max-abs {err.max():.3e} (excess {excess.max():.3e}) > {tol_max}"
@@ -67,7 +76,11 @@ def fwd_case(B, T, Hq, Hkv, D, sink, local, seed=50, windows=None, full_attn=Fal
 
 def test_fwd_tiny_config():
     c = cowa_inputs.CONFIGS["tiny"]
-    fwd_case(c["B"], c["T"], c["Hq"], c["Hkv"], c["D"], c["sink"], c["local"], seed=c["index"])
+    _CONFIG[0] = "tiny"
+    try:
+        fwd_case(c["B"], c["T"], c["Hq"], c["Hkv"], c["D"], c["sink"], c["local"], seed=c["index"])
+    finally:
+        _CONFIG[0] = None
 
 
 @pytest.mark.parametrize("B,T,Hq,Hkv,D,sink,local", [
@@ -102,11 +115,13 @@ def test_fwd_8k_config_sampled_heads():
     o, lse = run_fwd(q.to(DEV), k.to(DEV), v.to(DEV), params)
     ws = orc.default_windows(T, Hkv, c["sink"], c["local"])
     rows = np.arange(T)
+    _CONFIG[0] = "8k"
     for b, h in [(0, 0), (0, 7), (1, 9), (1, 15)]:
         o_ref, lse_ref = orc.forward_rows(cowa_inputs.to_f64(q[b]), cowa_inputs.to_f64(k[b]),
                                           cowa_inputs.to_f64(v[b]), ws, scale, h, rows)
         check(f"lse[{b},{h}]", lse[b, h].cpu().numpy(), lse_ref, TOL_LSE, TOL_LSE)
         check(f"o[{b},{h}]", o[b, h].float().cpu().numpy(), o_ref)
+    _CONFIG[0] = None
     # duplicated-window control at the same shape: one head pair
     wd = orc.duplicated_windows(T, Hkv, c["sink"], c["local"], 1)
     pd = cowa.make_params(softmax_scale=scale, windows=wd)
@@ -275,7 +290,11 @@ def bwd_case(B, T, Hq, Hkv, D, sink, local, seed=51, windows=None, full_attn=Fal
 
 def test_bwd_tiny_config():
     c = cowa_inputs.CONFIGS["tiny"]
-    bwd_case(c["B"], c["T"], c["Hq"], c["Hkv"], c["D"], c["sink"], c["local"], seed=c["index"])
+    _CONFIG[0] = "tiny"
+    try:
+        bwd_case(c["B"], c["T"], c["Hq"], c["Hkv"], c["D"], c["sink"], c["local"], seed=c["index"])
+    finally:
+        _CONFIG[0] = None
 
 
 @pytest.mark.parametrize("B,T,Hq,Hkv,D,sink,local", [
@@ -384,6 +403,7 @@ def test_bwd_8k_config_sampled():
     ws = orc.default_windows(T, Hkv, c["sink"], c["local"])
     f = cowa_inputs.to_f64
     # dQ: whole heads; dK/dV: KV tiles incl. the sink tile, a band edge and the last tile
+    _CONFIG[0] = "8k"
     for b, h in [(0, 1), (1, 14)]:
         ref = orc.backward_dq_rows(f(q[b]), f(k[b]), f(v[b]), f(d_o[b]), ws, scale, h, np.arange(T))
         check_grad(f"dq[{b},{h}]", dq[b, h].float().cpu().numpy(), ref)
@@ -392,6 +412,30 @@ def test_bwd_8k_config_sampled():
         dk_r, dv_r = orc.backward_dkdv_cols(f(q[b]), f(k[b]), f(v[b]), f(d_o[b]), ws, scale, hk, cols)
         check_grad(f"dk[{b},{hk},{tile}]", dk[b, hk, cols].float().cpu().numpy(), dk_r)
         check_grad(f"dv[{b},{hk},{tile}]", dv[b, hk, cols].float().cpu().numpy(), dv_r)
+    _CONFIG[0] = None
+
+
+def test_bwd_8k_duplicated_window_control():
+    """The 8K configuration's control layout (Sec. 3, "Collective Coverage with Matched Per-Head Window
+    Widths"): every KV head gets the band next to the near window (m = 1), passed as explicit tuples."""
+    c = cowa_inputs.CONFIGS["8k"]
+    B, T, Hq, Hkv, D = c["B"], c["T"], c["Hq"], c["Hkv"], c["D"]
+    q, k, v, d_o = cowa_inputs.make_train_inputs(c["index"], B, T, Hq, Hkv, D)
+    scale = cowa_inputs.softmax_scale(D)
+    wd = orc.duplicated_windows(T, Hkv, c["sink"], c["local"], 1)
+    params = cowa.make_params(softmax_scale=scale, windows=wd)
+    dq, dk, dv = run_fwd_bwd(q.to(DEV), k.to(DEV), v.to(DEV), d_o.to(DEV), params)
+    f = cowa_inputs.to_f64
+    _CONFIG[0] = "8k control"
+    b, h = 1, 6
+    ref = orc.backward_dq_rows(f(q[b]), f(k[b]), f(v[b]), f(d_o[b]), wd, scale, h, np.arange(T))
+    check_grad(f"dq[{b},{h}]", dq[b, h].float().cpu().numpy(), ref)
+    for b, hk, tile in [(0, 3, 0), (1, 2, 41)]:  # the sink tile and a tile whose queries straddle the band's far edge
+        cols = np.arange(tile * 128, tile * 128 + 128)
+        dk_r, dv_r = orc.backward_dkdv_cols(f(q[b]), f(k[b]), f(v[b]), f(d_o[b]), wd, scale, hk, cols)
+        check_grad(f"dk[{b},{hk},{tile}]", dk[b, hk, cols].float().cpu().numpy(), dk_r)
+        check_grad(f"dv[{b},{hk},{tile}]", dv[b, hk, cols].float().cpu().numpy(), dv_r)
+    _CONFIG[0] = None
 
 
 # ------------------------------------------------------------------ full-size configurations, sampled
@@ -424,6 +468,7 @@ def _full_size_sampled(name, q_tiles, kv_samples):
             cache[hk] = (f(k[0, hk:hk + 1]), f(v[0, hk:hk + 1]))
         return f(q[0, h:h + 1]), cache[hk][0], cache[hk][1], f(d_o[0, h:h + 1]), [ws[hk]]
 
+    _CONFIG[0] = name
     for h, tile in q_tiles:
         rows = np.arange(tile * 128, tile * 128 + 128)
         qh, kh, vh, doh, w1 = head_inputs(h)
@@ -438,6 +483,7 @@ def _full_size_sampled(name, q_tiles, kv_samples):
         dk_r, dv_r = orc.backward_dkdv_cols(qg, f(k[0, hk:hk + 1]), f(v[0, hk:hk + 1]), dog, [ws[hk]], scale, 0, cols)
         check_grad(f"{name} dk[hk{hk},tile{tile}]", dk[0, hk, cols].float().cpu().numpy(), dk_r)
         check_grad(f"{name} dv[hk{hk},tile{tile}]", dv[0, hk, cols].float().cpu().numpy(), dv_r)
+    _CONFIG[0] = None
 
 
 # ------------------------------------------------------------------ backward with N_q < N_k
@@ -551,8 +597,11 @@ def test_32k_config_sampled():
 
 
 def test_128k_config_sampled():
+    # KV tiles: one in the middle of a far head's range, the sink tile (the longest block of the launch: every
+    # query tile of the group's four heads visits it) and the tile of head 0 whose queries straddle the far
+    # edge of that head's band (near + band = 4096 + 15856 keys back)
     _full_size_sampled("128k", q_tiles=[(0, 1023), (5, 33), (13, 500), (31, 1023), (18, 157)],
-                       kv_samples=[(6, 901)])
+                       kv_samples=[(6, 901), (0, 0), (0, 867)])
 
 
 def test_one_million_tokens_sampled():
@@ -654,8 +703,37 @@ def test_decode_128k_config():
             qf = q[b:b + 1, hk * G:(hk + 1) * G].cpu().to(torch.float64).numpy()
             o_ref, lse_ref = orc.decode(qf, kf, vf, lens_h[b:b + 1], c["sink"], c["local"], scale,
                                         h_k_global=c["Hkv"], hk_offset=hk)
-            check(f"decode lse[{b},{hk}]", lse_h[b, hk * G:(hk + 1) * G], lse_ref[0], TOL_LSE, TOL_LSE)
-            check(f"decode o[{b},{hk}]", o_h[b, hk * G:(hk + 1) * G], o_ref[0])
+            _CONFIG[0] = "decode128k"
+            check(f"decode128k lse[{b},{hk}]", lse_h[b, hk * G:(hk + 1) * G], lse_ref[0], TOL_LSE, TOL_LSE)
+            check(f"decode128k o[{b},{hk}]", o_h[b, hk * G:(hk + 1) * G], o_ref[0])
+            _CONFIG[0] = None
+
+
+@pytest.mark.parametrize("offset,local_heads", [(0, 2), (3, 1), (7, 1), (5, 2)])
+def test_fwd_and_decode_with_global_head_offsets(offset, local_heads):
+    """A tensor-parallel rank holds KV heads offset .. offset+local_heads-1 of 8 and must use the windows of
+    the global head index (Eq. fwa_global_head; Sec. 2.3 "Global KV-head assignment"): forward O / LSE and
+    decode against the oracle evaluated with the same offset."""
+    T, G, D, sink, local = 2500, 4, 128, 24, 160
+    Hkv, Hq = local_heads, local_heads * G
+    scale = cowa_inputs.softmax_scale(D)
+    q, k, v, _ = cowa_inputs.make_train_inputs(90 + offset, 1, T, Hq, Hkv, D)
+    params = cowa.make_params(sink=sink, local=local, softmax_scale=scale, hkv_global=8, hkv_offset=offset)
+    o, lse = run_fwd(q.to(DEV), k.to(DEV), v.to(DEV), params)
+    ws = orc.default_windows(T, 8, sink, local, offset, local_heads)
+    assert ws == orc.default_windows(T, 8, sink, local)[offset:offset + local_heads]
+    f = cowa_inputs.to_f64
+    o_ref, lse_ref = orc.forward(f(q[0]), f(k[0]), f(v[0]), ws, scale)
+    check(f"shard {offset} lse", lse[0].cpu().numpy(), lse_ref, TOL_LSE, TOL_LSE)
+    check(f"shard {offset} o", o[0].float().cpu().numpy(), o_ref)
+    # decode over the same tensors used as a cache, two sequences of different lengths
+    lens = [T, 1777]
+    qd = torch.stack([q[0, :, n - 1] for n in lens]).contiguous()
+    kc, vc = k.expand(2, -1, -1, -1).contiguous(), v.expand(2, -1, -1, -1).contiguous()
+    o_d, lse_d = run_decode(qd.to(DEV), kc.to(DEV), vc.to(DEV), torch.tensor(lens, dtype=torch.int32, device=DEV), params)
+    od_ref, lsed_ref = orc.decode(f(qd), f(kc), f(vc), np.asarray(lens), sink, local, scale, h_k_global=8, hk_offset=offset)
+    check(f"shard {offset} decode lse", lse_d.cpu().numpy(), lsed_ref, TOL_LSE, TOL_LSE)
+    check(f"shard {offset} decode o", o_d.float().cpu().numpy(), od_ref)
 
 
 def test_decode_equals_last_forward_row():

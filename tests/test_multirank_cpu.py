@@ -75,3 +75,50 @@ def test_two_ranks_agree_on_global_heads_and_timing():
     r1 = [r for r in results if r[0] == "rank1"][0]
     assert r0[0] and r0[1]
     assert r0[2] == 11.0 and r1[1] == 11.0
+
+
+def _tp_worker(rank, world, port, out):
+    """bench.py --tp-replica under N processes: which TP=8 shards each process times, and the reduction of the
+    per-phase slowest shard over the processes (made-up latencies stand in for the GPU timings)."""
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        shards = bench.tp_shards(rank, world, 8)
+        # shard r "takes" 10 + r ms forward and 30 - r ms backward at one length, so the slowest forward shard is
+        # 7 and the slowest backward shard is 0, whoever owns them
+        row = {"T": 4096, "cowa_fwd_ms": max([10.0 + r for r in shards], default=0.0),
+               "cowa_bwd_ms": max([30.0 - r for r in shards], default=0.0)}
+        reduced = bench.reduce_worst([row], world)
+        gathered = [None] * world
+        dist.all_gather_object(gathered, shards)
+        out.put((rank, gathered, reduced))
+    finally:
+        dist.destroy_process_group()
+
+
+def _run_tp(world):
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_tp_worker, args=(r, world, port, out)) for r in range(world)]
+    for p in procs:
+        p.start()
+    results = [out.get(timeout=180) for _ in range(world)]
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    return results
+
+
+def test_tp_replica_shard_assignment_and_worst_shard_reduction():
+    for world in (2, 8):
+        for rank, gathered, reduced in _run_tp(world):
+            # every shard of the TP=8 group is timed by exactly one process; with 8 processes one each
+            assert sorted(s for g in gathered for s in g) == list(range(8))
+            assert gathered[rank] == list(range(rank, 8, world))
+            if world == 8:
+                assert all(len(g) == 1 for g in gathered)
+            # every process ends up with the group's latency: the slowest shard per phase
+            assert reduced == [{"T": 4096, "cowa_bwd_ms": 30.0, "cowa_fwd_ms": 17.0}]
+    assert bench.tp_shards(9, 16, 8) == []  # surplus processes own nothing

@@ -110,6 +110,9 @@ def test_mask_brute_force():
                 sink = ik < w[0] and d >= 0
                 far = w[1] + w[2] <= d < w[1] + w[2] + w[3]
                 assert m[iq, ik] == (near or sink or far)
+        # the mask restricted to chosen rows and key columns is the same predicate on that sub-rectangle
+        rows, cols = np.array([0, 5, 22]), np.array([40, 0, 7, 8, 33])
+        assert (orc.visible_mask(n_q, n_k, w, rows, cols) == m[np.ix_(rows, cols)]).all()
 
 
 def test_breakpoints_floor_and_global_index():

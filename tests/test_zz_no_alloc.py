@@ -10,6 +10,7 @@ import torch
 
 import cowa_inputs
 import paper_2609_32704_b200 as cowa
+from oracle import cowa_oracle as orc
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -41,11 +42,14 @@ def test_decode_static_matches_decode_on_two_calls_in_a_row():
         (71, 3, 6000, 8, 2, 128, 16, 200, [6000, 1, 3333]),
         (72, 2, 2500, 8, 8, 64, 4, 50, [2500, 999]),
     ]
-    prepared = []
+    prepared, oracle_out = [], []
     for seed, B, Tmax, Hq, Hkv, D, sink, local, lens in cases:
         params = cowa.make_params(sink=sink, local=local, softmax_scale=cowa_inputs.softmax_scale(D))
         t = _inputs(seed, B, Tmax, Hq, Hkv, D, lens)
         prepared.append((t, params, _reference(*t, params)))
+        q, kc, vc, ln = (x.cpu() for x in t)
+        oracle_out.append(orc.decode(cowa_inputs.to_f64(q), kc.float().numpy(), vc.float().numpy(), ln.numpy(),
+                                     sink, local, cowa_inputs.softmax_scale(D)))
     outs = []
     for (q, kc, vc, lens), params, _ in prepared:  # back to back on one stream, no sync between
         o = torch.full_like(q, float("nan"))
@@ -53,10 +57,13 @@ def test_decode_static_matches_decode_on_two_calls_in_a_row():
         cowa.cowa_decode_static(q, kc, vc, lens, o, lse, params)
         outs.append((o, lse))
     torch.cuda.synchronize()
-    for (o, lse), (_, _, (o_ref, lse_ref)) in zip(outs, prepared):
+    for (o, lse), (_, _, (o_ref, lse_ref)), (o_orc, lse_orc) in zip(outs, prepared, oracle_out):
         assert torch.isfinite(o.float()).all() and torch.isfinite(lse).all()
         assert (o.float() - o_ref.float()).abs().max().item() <= 2e-2
         assert (lse - lse_ref).abs().max().item() <= 1e-3
+        # and against the float64 oracle, like every other decode test
+        assert abs(o.float().cpu().numpy() - o_orc).max() <= 2e-2
+        assert abs(lse.cpu().numpy() - lse_orc).max() <= 1e-3
 
 
 def test_decode_static_rejects_oversized_calls():
