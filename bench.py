@@ -372,6 +372,26 @@ def run_cuda(args):
     barrier(world)
     dec_b2b_ms = max_over_ranks(eb[0].elapsed_time(eb[1]) / n_dec, world)
 
+    # ---- yardstick for the decode numbers: a plain streaming read of exactly as many bytes as the decode's
+    # visible K/V rows (a library reduction over a buffer of that size), timed in the same two situations: right
+    # behind a training backward, as inside the step, and back to back.  It shows what the GPU lets a pure read
+    # of these bytes do in that state (SM clock under the power cap, dirty L2 lines left by the backward).
+    yard = torch.ones(dec_bytes // 4, dtype=torch.float32, device=dev)
+    for _ in range(3):
+        yard.sum()
+    ey = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(4)]
+    for e_ in ey[:3]:
+        cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, p_train, ws_bwd)
+        e_[0].record(); yard.sum(); e_[1].record()
+    ey[3][0].record()
+    for _ in range(n_dec):
+        yard.sum()
+    ey[3][1].record()
+    torch.cuda.synchronize()
+    yard_step_ms = max_over_ranks(sum(e_[0].elapsed_time(e_[1]) for e_ in ey[:3]) / 3, world)
+    yard_b2b_ms = max_over_ranks(ey[3][0].elapsed_time(ey[3][1]) / n_dec, world)
+    del yard
+
     # ---- decode variants on the same cache: several newest tokens per call, paged cache ----
     dec_var = None
     if not args.no_varlen:
@@ -642,7 +662,11 @@ def run_cuda(args):
               "frac_nominal_8tbs": dec_gbs / 8000.0, "us_per_step_min": dec_min * 1e3,
               "back_to_back": {"us_per_call": dec_b2b_ms * 1e3, "achieved_gbs": b2b_gbs,
                                "frac_hbm": b2b_gbs / peaks["hbm_gbs"], "frac_nominal_8tbs": b2b_gbs / 8000.0,
-                               "calls": n_dec}}
+                               "calls": n_dec},
+              "plain_read_of_same_bytes": {"after_backward_us": yard_step_ms * 1e3, "back_to_back_us": yard_b2b_ms * 1e3,
+                                           "decode_over_read_in_step": dec_ms / yard_step_ms,
+                                           "decode_over_read_back_to_back": dec_b2b_ms / yard_b2b_ms,
+                                           "what": "torch.sum over a float32 buffer of visible_kv_bytes"}}
 
     cpu = None
     if not args.no_cpu_baseline and world == 1:  # the oracle is timed on one-GPU runs only

@@ -257,9 +257,12 @@ def backward_dq_rows(q, k, v, d_o, windows, scale, h, rows):
     return scale * (ds @ kc)
 
 
-def backward_dkdv_cols(q, k, v, d_o, windows, scale, hk, cols, row_block=1024):
+def backward_dkdv_cols(q, k, v, d_o, windows, scale, hk, cols, row_block=1024, row_range=None):
     """dK [C,D], dV [C,D] of KV head hk for the given key columns, summed over
-    the QO heads of the group and over every query row that sees any of them."""
+    the QO heads of the group and over every query row that sees any of them.
+    With row_range = (r0, r1) only the query rows r0 <= i_q < r1 are summed: the
+    gradients are sums over query rows, so the results of disjoint ranges add up
+    to the whole (a caller may walk the ranges in parallel)."""
     h_q, n_q, d = q.shape
     h_k, n_k, _ = k.shape
     cols = np.asarray(cols)
@@ -268,8 +271,9 @@ def backward_dkdv_cols(q, k, v, d_o, windows, scale, hk, cols, row_block=1024):
     dv = np.zeros((len(cols), v.shape[2]))
     kc_sel = np.asarray(k[hk][cols], dtype=np.float64)
     vc_sel = np.asarray(v[hk][cols], dtype=np.float64)
-    for r0 in range(0, n_q, row_block):
-        rows = np.arange(r0, min(r0 + row_block, n_q))
+    first, last = (0, n_q) if row_range is None else (max(int(row_range[0]), 0), min(int(row_range[1]), n_q))
+    for r0 in range(first, last, row_block):
+        rows = np.arange(r0, min(r0 + row_block, last))
         # rows that see none of the selected columns contribute nothing: find them from the mask on those
         # columns alone before the mask over all keys is built for the rest
         sel = visible_mask(n_q, n_k, windows[hk], rows, cols)

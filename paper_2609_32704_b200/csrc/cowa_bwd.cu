@@ -413,7 +413,7 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           }
         }
         // Step n uses TMEM buffer b = n & 1 (the two compute warpgroups alternate steps).  Issue order:
-        //   dV(n) | dP^T(n+1) | dK(n) | dQ^T(n) | S^T(n+2)
+        //   dV(n) | dP^T(n+1) | dK(n) | S^T(n+2) | dQ^T(n)
         // so that every wait below is for something produced about one step earlier.
         int st = 0, st1 = (N > 1) ? 1 : 0, st2 = 2 % NST;    // stages of steps n, n+1, n+2
         uint32_t ph2 = (2 / NST) & 1;                        // parity of the load that fills stage st2 for step n+2
@@ -439,15 +439,15 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           tc_fence_after();
           gemm_acc(cDK, sbuf + 16, dQ_mn0 + st * kStage16, n > 0 ? 1u : 0u);  // dK += dS^T Q
           commit(bar_ld_empty + st);
-          gemm_dq(dpbuf, dDS0 + b_ * kDS16);                                // dQ^T = K^T dS^T over the consumed dP^T(n)
-          commit(bar_dq_full + b_);
-          if (n + 2 < N) {                                                  // S^T(n+2) into the buffer P^T(n), dS^T(n) just left
-            ok = mbar_wait(bar_ld_full + st2, ph2, a.status);
-            if (!ok) return;
+          if (n + 2 < N) {                                                  // S^T(n+2) into the buffer P^T(n), dS^T(n) just left:
+            ok = mbar_wait(bar_ld_full + st2, ph2, a.status);               // it heads the next step's dependency chain, so it
+            if (!ok) return;                                                // goes ahead of dQ^T(n), which only feeds the drain
             tc_fence_after();
             gemm_st(sbuf, dK_k, dQ_k0 + st2 * kStage16);
             commit(bar_s_full + b_);
           }
+          gemm_dq(dpbuf, dDS0 + b_ * kDS16);                                // dQ^T = K^T dS^T over the consumed dP^T(n)
+          commit(bar_dq_full + b_);
           // advance the bookkeeping to step n+1
           st = st1; st1 = st2;
           if (++st2 == NST) { st2 = 0; ph2 ^= 1; }

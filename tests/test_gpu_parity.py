@@ -6,6 +6,8 @@ alone costs up to |x| * 2^-8 (half an ulp) and |x| * 2^-10 on average (a quarter
 least |x| * 2^-8); the gradient check therefore allows 2e-2 + 2^-8 * |reference| per element and
 2e-3 + 2^-10 * mean|reference| on average.  The second term only matters where most entries are
 large, e.g. a packed sequence of five tokens whose every key is attended with weight near one."""
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 import pytest
 import torch
@@ -480,7 +482,14 @@ def _full_size_sampled(name, q_tiles, kv_samples):
     for hk, tile in kv_samples:
         cols = np.arange(tile * 128, tile * 128 + 128)
         qg, dog = f(q[0, hk * G:(hk + 1) * G]), f(d_o[0, hk * G:(hk + 1) * G])
-        dk_r, dv_r = orc.backward_dkdv_cols(qg, f(k[0, hk:hk + 1]), f(v[0, hk:hk + 1]), dog, [ws[hk]], scale, 0, cols)
+        kg, vg = f(k[0, hk:hk + 1]), f(v[0, hk:hk + 1])
+        # dK, dV are sums over query rows: the oracle walks disjoint row ranges on the host's cores at once
+        # (numpy releases the interpreter lock) and the partial sums are added
+        edges = np.linspace(0, T, 17).astype(int)
+        with ThreadPoolExecutor(max_workers=8) as pool:
+            parts = list(pool.map(lambda r: orc.backward_dkdv_cols(qg, kg, vg, dog, [ws[hk]], scale, 0, cols,
+                                                                   row_range=(edges[r], edges[r + 1])), range(16)))
+        dk_r, dv_r = sum(x[0] for x in parts), sum(x[1] for x in parts)
         check_grad(f"{name} dk[hk{hk},tile{tile}]", dk[0, hk, cols].float().cpu().numpy(), dk_r)
         check_grad(f"{name} dv[hk{hk},tile{tile}]", dv[0, hk, cols].float().cpu().numpy(), dv_r)
     _CONFIG[0] = None

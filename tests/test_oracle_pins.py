@@ -326,6 +326,11 @@ def test_backward_vs_autograd_and_row_col_variants():
     dk_c, dv_c = orc.backward_dkdv_cols(q, k, v, d_o, ws, scale, 0, cols, row_block=7)
     np.testing.assert_allclose(dk_c, dk[0, cols], atol=1e-12)
     np.testing.assert_allclose(dv_c, dv[0, cols], atol=1e-12)
+    # disjoint query-row ranges add up to the whole
+    parts = [orc.backward_dkdv_cols(q, k, v, d_o, ws, scale, 0, cols, row_block=7, row_range=r)
+             for r in ((0, 11), (11, 12), (12, n_q))]
+    np.testing.assert_allclose(sum(x[0] for x in parts), dk[0, cols], atol=1e-12)
+    np.testing.assert_allclose(sum(x[1] for x in parts), dv[0, cols], atol=1e-12)
 
 
 # ---------------------------------------------------------------- decode
