@@ -42,8 +42,8 @@ def load_peaks():
 
 
 def load_traffic():
-    """DRAM bytes per launch of the kernels, from the tracked ncu summary file profiles/traffic.json:
-    {kernel name: {"bytes_per_launch": ..., "workload": ..., "source": ...}}.  Missing file or kernel: None."""
+    """DRAM bytes per launch of the kernels, from the tracked ncu summary profiles/traffic.json:
+    {kernel name: {workload: {"bytes_per_launch": ..., "source": ...}}}."""
     path = os.path.join(ROOT, "profiles", "traffic.json")
     if not os.path.exists(path):
         return {}
@@ -52,10 +52,12 @@ def load_traffic():
 
 
 def traffic_for(table, kernel, workload):
+    """The recorded figure for this kernel name and workload, or None: a renamed kernel or a workload that was
+    never captured gets no number."""
     e = table.get(kernel)
-    if not e or e.get("workload") != workload:
+    if not isinstance(e, dict) or workload not in e:
         return None
-    return e.get("bytes_per_launch")
+    return e[workload].get("bytes_per_launch")
 
 
 def tp_shards(rank, world, tp):
