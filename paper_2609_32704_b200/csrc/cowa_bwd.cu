@@ -394,10 +394,40 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           if (lead) mma_commit(bar);
         };
 
+        // Packed batches: rows of a tile that lie past the end of the sequence belong to the next one.  Every
+        // product they enter is multiplied by an exact zero, but 0 x (Inf or NaN) would still poison this
+        // sequence, so they are cleared in shared memory (whole 128-byte rows, by this warp) before use.
+        auto clear_rows = [&](uint8_t* tile, int first, int rows, int slab_bytes) {
+          const int nchunk = (rows - first) * 8;  // 16-byte chunks per slab
+          for (int s_ = 0; s_ < NSLAB; ++s_)
+            for (int c_ = lane; c_ < nchunk; c_ += 32)
+              *reinterpret_cast<uint4*>(tile + s_ * slab_bytes + first * 128 + c_ * 16) = make_uint4(0u, 0u, 0u, 0u);
+        };
+        int t_clr = 0;  // position in I_h(j) of the next step whose Q / dO stage is checked (packed batches only)
+        auto clear_stage_tail = [&](int stage) {
+          if constexpr (VARLEN) {
+            const int q0_ = cowa_bwd_tile_at(rg, t_clr) * BQS;
+            if (++t_clr == cnt) t_clr = 0;
+            if (q0_ + BQS > Nq) {
+              uint8_t* sQ_ = sStage + stage * SM::kStage;
+              clear_rows(sQ_, Nq - q0_, BQS, SLAB_QS);
+              clear_rows(sQ_ + SM::kQS, Nq - q0_, BQS, SLAB_QS);
+              fence_proxy_async_smem();
+              __syncwarp();
+            }
+          }
+        };
         ok = mbar_wait(bar_kv, 0, a.status);
+        if (ok && tail_kv) {
+          clear_rows(sK, Nk - k0, BKV, SLAB_KV);
+          clear_rows(sV, Nk - k0, BKV, SLAB_KV);
+          fence_proxy_async_smem();
+          __syncwarp();
+        }
         // prologue: S^T(0), dP^T(0), S^T(1)
         ok = ok && mbar_wait(bar_ld_full + 0, 0, a.status);
         if (ok) {
+          clear_stage_tail(0);
           tc_fence_after();
           gemm_st(cS0, dK_k, dQ_k0);
           commit(bar_s_full + 0);
@@ -407,6 +437,7 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (ok && N > 1) {
           ok = mbar_wait(bar_ld_full + 1, 0, a.status);
           if (ok) {
+            clear_stage_tail(1);
             tc_fence_after();
             gemm_st(cS0 + 64, dK_k, dQ_k0 + kStage16);
             commit(bar_s_full + 1);
@@ -442,6 +473,7 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           if (n + 2 < N) {                                                  // S^T(n+2) into the buffer P^T(n), dS^T(n) just left:
             ok = mbar_wait(bar_ld_full + st2, ph2, a.status);               // it heads the next step's dependency chain, so it
             if (!ok) return;                                                // goes ahead of dQ^T(n), which only feeds the drain
+            clear_stage_tail(st2);
             tc_fence_after();
             gemm_st(sbuf, dK_k, dQ_k0 + st2 * kStage16);
             commit(bar_s_full + b_);

@@ -358,6 +358,22 @@ cowa_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
       tmem_st32(t_S, pk);  // P over the first 32 columns of this S buffer
       tmem_wait_st();
+      if constexpr (VARLEN) {
+        // Last key tile of a packed sequence: the rows after it in shared memory belong to the next sequence.
+        // Their P entries are exactly zero, but 0 x (Inf or NaN) in the product would still poison this
+        // sequence, so those V rows are cleared before the product may start.
+        const int vrows = Nk - j * BK;  // valid rows of this 64-row tile
+        if (vrows < BK) {
+          ok = mbar_wait(bar_v + b_, (t >> 1) & 1, a.status);
+          if (!ok) break;
+          uint8_t* vt = sV + b_ * SM::kKV;
+          const int nchunk = (BK - vrows) * 8;  // 16-byte chunks per slab
+          for (int s_ = 0; s_ < NSLAB; ++s_)
+            for (int c_ = tid; c_ < nchunk; c_ += 128)
+              *reinterpret_cast<uint4*>(vt + s_ * SLAB_K + vrows * 128 + c_ * 16) = make_uint4(0u, 0u, 0u, 0u);
+          fence_proxy_async_smem();
+        }
+      }
       tc_fence_before();
       mbar_arrive(bar_p + b_);
       if (j > j_last) --j; else next_range();

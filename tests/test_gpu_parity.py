@@ -575,6 +575,42 @@ def test_bwd_varlen(lens, Hq, Hkv, D, sink, local, mode):
         check_grad(f"varlen dv[seq {b}]", dv[:, sl].float().cpu().numpy(), dv_r)
 
 
+@pytest.mark.parametrize("bad", [float("nan"), float("inf")])
+def test_packed_batch_nonfinite_neighbour_does_not_leak(bad):
+    """Rows past the end of a sequence share its last tiles in shared memory.  They are multiplied by exact
+    zeros, which is not enough when they hold Inf or NaN: a sequence's outputs must not depend on its
+    neighbour's values at all.  Sequence 1 is filled with non-finite values; sequences 0 and 2 must still match
+    the oracle (forward and backward), and sequence 1's own outputs are allowed to be anything."""
+    lens, Hq, Hkv, D, sink, local = [100, 300, 777], 4, 2, 128, 8, 40
+    seqs = [(n, n) for n in lens]
+    q, k, v, cu, _ = _packed_inputs(120, seqs, Hq, Hkv, D)
+    d_o = torch.cat([cowa_inputs.make_train_inputs(130 + b, 1, n, Hq, Hkv, D)[3][0] for b, n in enumerate(lens)], 1).contiguous()
+    sl1 = slice(int(cu[1]), int(cu[2]))
+    for t in (q, k, v, d_o):
+        t[:, sl1] = bad
+    scale = cowa_inputs.softmax_scale(D)
+    params = cowa.make_params(sink=sink, local=local, softmax_scale=scale)
+    o, lse = _run_varlen(q, k, v, cu, cu, params)
+    qd, kd, vd, dod = q.to(DEV), k.to(DEV), v.to(DEV), d_o.to(DEV)
+    dq, dk, dv = (torch.full_like(x, float("nan")) for x in (qd, kd, vd))
+    total = int(cu[-1])
+    ws = torch.empty(cowa.cowa_bwd_varlen_workspace_bytes(len(lens), total, Hq, Hkv, D, params), dtype=torch.uint8, device=DEV)
+    cowa.cowa_bwd_varlen(qd, kd, vd, o, lse, dod, dq, dk, dv, torch.from_numpy(cu).to(DEV), params, ws)
+    torch.cuda.synchronize()
+    cowa.cowa_check_device_status()
+    f = cowa_inputs.to_f64
+    for b in (0, 2):
+        sl = slice(int(cu[b]), int(cu[b + 1]))
+        wins = orc.default_windows(lens[b], Hkv, sink, local)
+        o_ref, lse_ref = orc.forward(f(q[:, sl]), f(k[:, sl]), f(v[:, sl]), wins, scale)
+        check(f"neighbour lse[{b}]", lse[:, sl].cpu().numpy(), lse_ref, TOL_LSE, TOL_LSE)
+        check(f"neighbour o[{b}]", o[:, sl].float().cpu().numpy(), o_ref)
+        dq_r, dk_r, dv_r = orc.backward(f(q[:, sl]), f(k[:, sl]), f(v[:, sl]), f(d_o[:, sl]), wins, scale)
+        check_grad(f"neighbour dq[{b}]", dq[:, sl].float().cpu().numpy(), dq_r)
+        check_grad(f"neighbour dk[{b}]", dk[:, sl].float().cpu().numpy(), dk_r)
+        check_grad(f"neighbour dv[{b}]", dv[:, sl].float().cpu().numpy(), dv_r)
+
+
 def test_bwd_varlen_equals_batched_dkdv():
     """Equal-length sequences: dK and dV of the packed call equal the batched call's bit for bit (same block
     arithmetic); dQ agrees within the tolerance (reduction order differs)."""
