@@ -374,26 +374,6 @@ def run_cuda(args):
     barrier(world)
     dec_b2b_ms = max_over_ranks(eb[0].elapsed_time(eb[1]) / n_dec, world)
 
-    # ---- yardstick for the decode numbers: a plain streaming read of exactly as many bytes as the decode's
-    # visible K/V rows (a library reduction over a buffer of that size), timed in the same two situations: right
-    # behind a training backward, as inside the step, and back to back.  It shows what the GPU lets a pure read
-    # of these bytes do in that state (SM clock under the power cap, dirty L2 lines left by the backward).
-    yard = torch.ones(dec_bytes // 4, dtype=torch.float32, device=dev)
-    for _ in range(3):
-        yard.sum()
-    ey = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(4)]
-    for e_ in ey[:3]:
-        cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, p_train, ws_bwd)
-        e_[0].record(); yard.sum(); e_[1].record()
-    ey[3][0].record()
-    for _ in range(n_dec):
-        yard.sum()
-    ey[3][1].record()
-    torch.cuda.synchronize()
-    yard_step_ms = max_over_ranks(sum(e_[0].elapsed_time(e_[1]) for e_ in ey[:3]) / 3, world)
-    yard_b2b_ms = max_over_ranks(ey[3][0].elapsed_time(ey[3][1]) / n_dec, world)
-    del yard
-
     # ---- decode variants on the same cache: several newest tokens per call, paged cache ----
     dec_var = None
     if not args.no_varlen:
@@ -437,6 +417,26 @@ def run_cuda(args):
                                   "max_abs_diff_vs_contiguous": float((o1.view_as(od).float() - od.float()).abs().max())}
         cowa.cowa_check_device_status()
         del kp, vp
+
+    # ---- yardstick for the decode numbers: a plain streaming read of exactly as many bytes as the decode's
+    # visible K/V rows (a library reduction over a buffer of that size), timed in the same two situations: right
+    # behind a training backward, as inside the step, and back to back.  It shows what the GPU lets a pure read
+    # of these bytes do in that state (SM clock under the power cap, dirty L2 lines left by the backward).
+    yard = torch.ones(dec_bytes // 4, dtype=torch.float32, device=dev)
+    for _ in range(3):
+        yard.sum()
+    ey = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(4)]
+    for e_ in ey[:3]:
+        cowa.cowa_bwd(q, k, v, o, lse, d_o, dq, dk, dv, p_train, ws_bwd)
+        e_[0].record(); yard.sum(); e_[1].record()
+    ey[3][0].record()
+    for _ in range(n_dec):
+        yard.sum()
+    ey[3][1].record()
+    torch.cuda.synchronize()
+    yard_step_ms = max_over_ranks(sum(e_[0].elapsed_time(e_[1]) for e_ in ey[:3]) / 3, world)
+    yard_b2b_ms = max_over_ranks(ey[3][0].elapsed_time(ey[3][1]) / n_dec, world)
+    del yard
 
     # ---- FullAttn path of the same library: the same step (forward, backward, decode in that order), one
     # warm-up step and three timed ones (it is ~5.4x the work), so that every ratio compares like with like ----
