@@ -574,8 +574,13 @@ def run_cuda(args):
         ho = torch.empty_like(hq).pin_memory()
         hlse = torch.empty(lse.shape, dtype=torch.float32).pin_memory()
         hdq, hdk, hdv = (torch.empty_like(x).pin_memory() for x in (hq, hk_, hv))
-        h2d = sum(x.numel() * x.element_size() for x in ((hq, hk_, hv, hdo) if have_bwd else (hq, hk_, hv)))
-        d2h = sum(x.numel() * x.element_size() for x in ((ho, hlse, hdq, hdk, hdv) if have_bwd else (ho, hlse)))
+        # decode step of the same pass: the query tokens come from the host and the outputs go back; the KV
+        # cache stays resident, as it does in a serving loop
+        hqd = qd.cpu().pin_memory()
+        hod = torch.empty_like(hqd).pin_memory()
+        qd2, od2 = torch.empty_like(qd), torch.empty_like(od)
+        h2d = sum(x.numel() * x.element_size() for x in (hq, hk_, hv, hdo, hqd))
+        d2h = sum(x.numel() * x.element_size() for x in (ho, hlse, hdq, hdk, hdv, hod))
 
         # Three streams (inputs, compute, results) and two sets of device buffers: PCIe is full duplex, and
         # as in a training loop that prefetches its next batch, the inputs of step s+1 come in while step s
@@ -618,7 +623,13 @@ def run_cuda(args):
                         s_out.wait_event(ev_bwd)
                         hdq.copy_(d["dq"], non_blocking=True); hdk.copy_(d["dk"], non_blocking=True)
                         hdv.copy_(d["dv"], non_blocking=True)
-                computed[s_ & 1] = ev_bwd if have_bwd else ev_fwd
+                # decode: 64 KB in, 64 KB out, on the compute stream itself (too small to be worth a stream hop)
+                qd2.copy_(hqd, non_blocking=True)
+                cowa.cowa_decode(qd2, kc, vc, lens, od2, lsed, p_dec, ws_dec)
+                hod.copy_(od2, non_blocking=True)
+                ev_step = torch.cuda.Event()
+                ev_step.record()
+                computed[s_ & 1] = ev_step
                 with torch.cuda.stream(s_out):
                     drained[s_ & 1] = torch.cuda.Event()
                     drained[s_ & 1].record()
@@ -634,8 +645,10 @@ def run_cuda(args):
         barrier(world)
         e_ms = max_over_ranks(ee[0].elapsed_time(ee[1]) / n_e2e, world)
         e2e = {"value": world * train_flops / (e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e_ms,
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e}
-        del hq, hk_, hv, hdo, ho, hlse, hdq, hdk, hdv, sets
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e,
+               "phases": ["fwd", "bwd", "decode"],
+               "note": "value = forward + backward FLOPs over the whole step time, decode step and all copies included"}
+        del hq, hk_, hv, hdo, ho, hlse, hdq, hdk, hdv, sets, hqd, hod, qd2, od2
 
     if rank != 0:
         return
