@@ -191,3 +191,41 @@ def test_deterministic_dq_out_of_range_is_reported():
         cowa.cowa_check_device_status()
     assert e.value.status == -9
     cowa.cowa_check_device_status()
+
+
+def test_prefill_and_its_backward_on_strided_views():
+    """N_q < N_k (a chunk appended to a cache) with q/o token-major and k/v slices of a wider cache buffer."""
+    B, Nq, Nk, Hq, Hkv, D, sink, local = 2, 200, 900, 8, 2, 128, 8, 90
+    q, _, _, d_o = cowa_inputs.make_train_inputs(101, B, Nq, Hq, Hkv, D)
+    _, k, v, _ = cowa_inputs.make_train_inputs(102, B, Nk, Hq, Hkv, D)
+    scale = cowa_inputs.softmax_scale(D)
+    params = cowa.make_params(sink=sink, local=local, softmax_scale=scale)
+    qs, dos = _bthd(q.to(DEV)), _bthd(d_o.to(DEV))
+    wide_k = torch.full((B, Hkv, Nk + 56, D), float("nan"), dtype=torch.bfloat16, device=DEV)
+    wide_v = torch.full_like(wide_k, float("nan"))
+    ks, vs = wide_k[:, :, 24:24 + Nk], wide_v[:, :, 24:24 + Nk]   # 16-byte aligned start, batch / head strides of the wide buffer
+    ks.copy_(k.to(DEV)); vs.copy_(v.to(DEV))
+    assert not ks.is_contiguous()
+    o = _bthd(torch.full((B, Hq, Nq, D), float("nan"), dtype=torch.bfloat16, device=DEV))
+    lse = torch.full((B, Hq, Nq), float("nan"), dtype=torch.float32, device=DEV)
+    cowa.cowa_prefill(qs, ks, vs, o, lse, params)
+    dq = _bthd(torch.full((B, Hq, Nq, D), float("nan"), dtype=torch.bfloat16, device=DEV))
+    wide_dk, wide_dv = torch.zeros_like(wide_k), torch.zeros_like(wide_v)
+    dk, dv = wide_dk[:, :, 24:24 + Nk], wide_dv[:, :, 24:24 + Nk]
+    ws = torch.empty(cowa.cowa_bwd_prefill_workspace_bytes(B, Nq, Nk, Hq, Hkv, D, params), dtype=torch.uint8, device=DEV)
+    cowa.cowa_bwd_prefill(qs, ks, vs, o, lse, dos, dq, dk, dv, params, ws)
+    torch.cuda.synchronize()
+    cowa.cowa_check_device_status()
+    # nothing outside the slices was written
+    assert (wide_dk[:, :, :24] == 0).all() and (wide_dk[:, :, 24 + Nk:] == 0).all()
+    assert (wide_dv[:, :, :24] == 0).all() and (wide_dv[:, :, 24 + Nk:] == 0).all()
+    wins = orc.default_windows(Nk, Hkv, sink, local)
+    f = cowa_inputs.to_f64
+    for b in range(B):
+        o_ref, lse_ref = orc.forward(f(q[b]), f(k[b]), f(v[b]), wins, scale)
+        _check(f"prefill lse[{b}]", lse[b].cpu().numpy(), lse_ref, TOL_LSE, TOL_LSE)
+        _check(f"prefill o[{b}]", o[b].float().cpu().numpy(), o_ref)
+        dq_r, dk_r, dv_r = orc.backward(f(q[b]), f(k[b]), f(v[b]), f(d_o[b]), wins, scale)
+        _check(f"prefill dq[{b}]", dq[b].float().cpu().numpy(), dq_r, grad=True)
+        _check(f"prefill dk[{b}]", dk[b].float().cpu().numpy(), dk_r, grad=True)
+        _check(f"prefill dv[{b}]", dv[b].float().cpu().numpy(), dv_r, grad=True)
