@@ -98,3 +98,26 @@ def test_scale_and_window_arguments():
     assert cowa.cowa_schedule_dump(cowa.SCHED_FWD, 512, 512, HKV, p) == \
         cowa.cowa_schedule_dump(cowa.SCHED_FWD, 512, 512, HKV, ref)
     assert cowa.cowa_tile_counts(512, 512, HKV, p) == cowa.cowa_tile_counts(512, 512, HKV, ref)
+
+
+def test_params_struct_layout_matches_the_header(tmp_path):
+    """The ctypes mirror of cowa_params_t must have the C compiler's layout of the struct in include/cowa.h."""
+    import os
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("no C compiler")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    fields = [n for n, _ in cowa.Params._fields_]
+    prog = ['#include <stdio.h>', '#include <stddef.h>', '#include "cowa.h"', 'int main(void) {',
+            '  printf("%zu\\n", sizeof(cowa_params_t));']
+    prog += [f'  printf("%zu\\n", offsetof(cowa_params_t, {n}));' for n in fields]
+    prog += ['  printf("%zu\\n", sizeof(cowa_window_t));', '  return 0;', '}']
+    src = tmp_path / "layout.c"
+    src.write_text("\n".join(prog))
+    exe = tmp_path / "layout"
+    subprocess.check_call(["gcc", "-std=c99", "-I", os.path.join(root, "include"), "-o", str(exe), str(src)])
+    out = [int(x) for x in subprocess.check_output([str(exe)]).split()]
+    assert out[0] == C.sizeof(cowa.Params)
+    assert out[1:-1] == [getattr(cowa.Params, n).offset for n in fields]
+    assert out[-1] == C.sizeof(cowa.Window)
