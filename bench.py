@@ -578,7 +578,8 @@ def run_cuda(args):
         # cache stays resident, as it does in a serving loop
         hqd = qd.cpu().pin_memory()
         hod = torch.empty_like(hqd).pin_memory()
-        qd2, od2 = torch.empty_like(qd), torch.empty_like(od)
+        qd2 = [torch.empty_like(qd) for _ in range(2)]
+        od2 = [torch.empty_like(od) for _ in range(2)]
         h2d = sum(x.numel() * x.element_size() for x in (hq, hk_, hv, hdo, hqd))
         d2h = sum(x.numel() * x.element_size() for x in (ho, hlse, hdq, hdk, hdv, hod))
 
@@ -602,6 +603,8 @@ def run_cuda(args):
                 with torch.cuda.stream(s_in):
                     if computed[s_ & 1] is not None:
                         s_in.wait_event(computed[s_ & 1]); s_in.wait_event(drained[s_ & 1])
+                    # the decode step's query tokens first: 64 KB that must not queue behind gigabytes on the copy engine
+                    qd2[s_ & 1].copy_(hqd, non_blocking=True)
                     d["q"].copy_(hq, non_blocking=True); d["k"].copy_(hk_, non_blocking=True)
                     d["v"].copy_(hv, non_blocking=True)
                     ev_qkv.record()
@@ -623,14 +626,14 @@ def run_cuda(args):
                         s_out.wait_event(ev_bwd)
                         hdq.copy_(d["dq"], non_blocking=True); hdk.copy_(d["dk"], non_blocking=True)
                         hdv.copy_(d["dv"], non_blocking=True)
-                # decode: 64 KB in, 64 KB out, on the compute stream itself (too small to be worth a stream hop)
-                qd2.copy_(hqd, non_blocking=True)
-                cowa.cowa_decode(qd2, kc, vc, lens, od2, lsed, p_dec, ws_dec)
-                hod.copy_(od2, non_blocking=True)
+                # decode on the resident cache; its 64 KB of output leave on the result stream with the gradients
+                cowa.cowa_decode(qd2[s_ & 1], kc, vc, lens, od2[s_ & 1], lsed, p_dec, ws_dec)
                 ev_step = torch.cuda.Event()
                 ev_step.record()
                 computed[s_ & 1] = ev_step
                 with torch.cuda.stream(s_out):
+                    s_out.wait_event(ev_step)
+                    hod.copy_(od2[s_ & 1], non_blocking=True)
                     drained[s_ & 1] = torch.cuda.Event()
                     drained[s_ & 1].record()
             s_main.wait_stream(s_in); s_main.wait_stream(s_out)
