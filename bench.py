@@ -159,36 +159,64 @@ def max_over_ranks(x, world):
 # ------------------------------------------------------------------------------------------
 
 def oracle_sample(budget_s, seed_tiles=0):
-    """Times the oracle's forward on whole 128-row query tiles of the 128K configuration, one
-    (head, tile) at a time, until about budget_s seconds are spent.  Returns FLOPs over legal
-    pairs (4*D per pair) and the seconds used."""
+    """Times the oracle on units of the 128K training configuration until about budget_s seconds are spent.
+    A unit is one (KV head, 128-row query tile): its forward (O, LSE) and the backward terms that belong to
+    those query rows (recompute of S and P, dP, dS, dQ); the dK / dV sums of a unit's keys run over every query
+    row of the sequence and are left out of the sample.  Returns the FLOPs the oracle actually performed over
+    legal pairs (4*D per pair forward, 6*D per pair for S, dP and dQ of the backward), the seconds used and the
+    number of units."""
     import numpy as np
     import torch
     import cowa_inputs
     from oracle import cowa_oracle as orc
     c = cowa_inputs.CONFIGS[TRAIN_CFG]
     T, Hq, Hkv, D = c["T"], c["Hq"], c["Hkv"], c["D"]
-    G = Hq // Hkv
     ws = orc.default_windows(T, Hkv, c["sink"], c["local"])
     scale = cowa_inputs.softmax_scale(D)
     g = torch.Generator().manual_seed(c["index"] * 1000 + 7)
-    # one KV head's tensors (synthetic N(0,1), bf16-rounded like the GPU inputs), reused by every sample
+    # one head's tensors (synthetic N(0,1), bf16-rounded like the GPU inputs), reused by every unit
     flops, secs, units = 0.0, 0.0, 0
     rng = np.random.default_rng(seed_tiles)
     k = torch.randn(1, T, D, generator=g).to(torch.bfloat16).to(torch.float64).numpy()
     v = torch.randn(1, T, D, generator=g).to(torch.bfloat16).to(torch.float64).numpy()
     q = torch.randn(1, T, D, generator=g).to(torch.bfloat16).to(torch.float64).numpy()
+    d_o = torch.randn(1, T, D, generator=g).to(torch.bfloat16).to(torch.float64).numpy()
     while secs < budget_s:
         hk = int(rng.integers(0, Hkv))
         tile = int(rng.integers(0, T // 128))
         rows = np.arange(tile * 128, tile * 128 + 128)
         t0 = time.perf_counter()
         orc.forward_rows(q, k, v, [ws[hk]], scale, 0, rows)
+        orc.backward_dq_rows(q, k, v, d_o, [ws[hk]], scale, 0, rows)
         secs += time.perf_counter() - t0
         pairs = int(orc.visible_mask(T, T, ws[hk], rows).sum())
-        flops += 4.0 * D * pairs
+        flops += (4.0 + 6.0) * D * pairs
         units += 1
     return flops, secs, units
+
+
+def oracle_decode_sample(reps=3):
+    """Times the oracle's decode of one (sequence, KV head) of the 128K decode configuration: visible K/V bytes
+    per second of host time (what the GPU path reports for the whole batch)."""
+    import numpy as np
+    import torch
+    import cowa_inputs
+    from oracle import cowa_oracle as orc
+    c = cowa_inputs.CONFIGS[DECODE_CFG]
+    D, G = c["D"], c["Hq"] // c["Hkv"]
+    n_k = (c["len_lo"] + c["len_hi"]) // 2
+    g = torch.Generator().manual_seed(c["index"] * 1000 + 9)
+    kc = torch.randn(1, 1, n_k, D, generator=g).to(torch.bfloat16).to(torch.float64).numpy()
+    vc = torch.randn(1, 1, n_k, D, generator=g).to(torch.bfloat16).to(torch.float64).numpy()
+    qd = torch.randn(1, G, D, generator=g).to(torch.bfloat16).to(torch.float64).numpy()
+    lens = np.array([n_k])
+    win = orc.default_windows(n_k, c["Hkv"], c["sink"], c["local"])[3]
+    vis = int(orc.visible_mask(1, n_k, win).sum())
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        orc.decode(qd, kc, vc, lens, c["sink"], c["local"], cowa_inputs.softmax_scale(D), h_k_global=c["Hkv"], hk_offset=3)
+    dt = (time.perf_counter() - t0) / reps
+    return vis * D * 2 * 2 / dt / 1e9, dt
 
 
 def count_legal_pairs(T, windows):
@@ -237,8 +265,9 @@ def run_reference(args):
         f, t, _ = oracle_sample(per_step, seed_tiles=s)
         flops, secs = flops + f, secs + t
     val = flops / secs / 1e12
-    sample = (f"oracle forward on random (KV head, 128-row query tile) samples of the 128K configuration, "
-              f"~{per_step:.0f} s per step")
+    sample = (f"oracle forward + the backward terms of the same query rows (S, P, dP, dS, dQ; dK/dV not sampled) on "
+              f"random (KV head, 128-row query tile) units of the 128K configuration, ~{per_step:.0f} s per step; "
+              f"FLOPs as performed over legal pairs (10*D per pair)")
     line = {
         "impl": "reference", "metric": "cowa_train_tflops_visited_tiles_128k", "value": val, "unit": "TFLOP/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / args.steps,
@@ -689,9 +718,13 @@ def run_cuda(args):
     cpu = None
     if not args.no_cpu_baseline and world == 1:  # the oracle is timed on one-GPU runs only
         f, t, units = oracle_sample(args.cpu_seconds)
+        dec_gbs_cpu, dec_s_cpu = oracle_decode_sample()
         cpu = {"value": f / t / 1e12, "unit": "TFLOP/s", "cores": cpu_threads(), "kind": "oracle",
-               "sample": f"oracle forward of {units} random (KV head, 128-row query tile) units of the 128K "
-                         f"configuration, {t:.1f} s; legal-pair FLOPs"}
+               "sample": f"oracle forward + the backward terms of the same query rows (S, P, dP, dS, dQ; dK/dV sums run "
+                         f"over all query rows and are not sampled) of {units} random (KV head, 128-row query tile) units "
+                         f"of the 128K configuration, {t:.1f} s; FLOPs as performed over legal pairs (10*D per pair)",
+               "decode": {"value": dec_gbs_cpu, "unit": "GB/s of visible K/V", "seconds_per_sequence_and_kv_head": dec_s_cpu,
+                          "sample": "oracle decode of one (sequence, KV head) of the 128K decode configuration"}}
 
     line = {
         "metric": "cowa_train_tflops_visited_tiles_" + args.train_cfg, "value": value, "unit": "TFLOP/s", "n_gpus": world,
