@@ -15,7 +15,7 @@
 //                   dK and dV stay in TMEM for the whole loop, all G heads included, so they need no
 //                   atomics (Algorithm 2 line 17 needs them only because it gives each QO head its
 //                   own program).  dQ^T is drained by a separate warpgroup through shared memory and
-//                   added to the fp32 accumulator with TMA bulk reductions (Algorithm 2 line 15).
+//                   added to the fp32 accumulator with bulk add-reductions of contiguous 32-row ranges (Algorithm 2 line 15).
 //                   Warp roles: TMA producer / MMA issuer / two compute warpgroups (P, dS; each takes 32
 //                   of the 64 query columns of every step, which halves the latency between S^T and
 //                   dS^T) / dQ drain warpgroup, connected by mbarriers; S^T is double buffered so that the
@@ -107,7 +107,7 @@ __global__ void __launch_bounds__(512, 1)
 cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmdO,
                 const __grid_constant__ CUtensorMap tmdK, const __grid_constant__ CUtensorMap tmdV,
-                const __grid_constant__ CUtensorMap tmdQ, const __grid_constant__ BwdArgs a) {
+                const __grid_constant__ BwdArgs a) {
   using SM = BwdSmem<D>;
   constexpr int NSLAB = D / 64;
   constexpr int SLAB_KV = BKV * 128;  // bytes of one 64-wide slab of a 128-row tile
@@ -630,7 +630,10 @@ cowa_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           fence_proxy_async_smem();
           wg_sync(3);
           if (issuer) {
-            tma_reduce_add_4d(&tmdQ, stage, 0, pbase + q0 + hf * 32, bhq, 0);
+            // 32 query rows of the accumulator are one contiguous range (rows are D floats, padded row space)
+            void* gdst = a.dq_acc + (((size_t)bhq * vec_stride + pbase + q0 + hf * 32) * D);
+            if (a.dq_fixed) bulk_reduce_add_s32(gdst, stage, 32 * D * 4);
+            else bulk_reduce_add_f32(gdst, stage, 32 * D * 4);
             tma_commit_group();
           }
         }
@@ -891,10 +894,7 @@ int launch_bwd(const void* q, const void* k, const void* v, const void* o, const
   if ((rc = cowa::resolve_strides(p->v_strides, Hkv, Nk, D, &sv))) return rc;
   if ((rc = cowa::resolve_strides(p->o_strides, Hq, Nq, D, &so))) return rc;
   if (BH > 0x7FFFFFFFll) return COWA_ERR_UNSUPPORTED;
-  CUtensorMap mq, mk, mv, mdo, mdk, mdv, mdq;
-  if ((rc = cowa::make_tensor_map(&mdq, dq_acc, p->deterministic ? cowa::MapType::S32 : cowa::MapType::F32, D, Tpad, (int)BH,
-                                  1, packed_strides((int)BH, Tpad, D), D, 32, false)))
-    return rc;
+  CUtensorMap mq, mk, mv, mdo, mdk, mdv;
   if ((rc = cowa::make_tensor_map(&mq, q, cowa::MapType::BF16, D, T, Hq, B, sq, 64, BQS))) return rc;
   if ((rc = cowa::make_tensor_map(&mdo, d_o, cowa::MapType::BF16, D, T, Hq, B, so, 64, BQS))) return rc;
   if ((rc = cowa::make_tensor_map(&mk, k, cowa::MapType::BF16, D, Nk, Hkv, B, sk, 64, BKV))) return rc;
@@ -930,7 +930,7 @@ int launch_bwd(const void* q, const void* k, const void* v, const void* o, const
     COWA_CUDA_TRY(cudaGetLastError());
   }
   if (p->bwd_main_start_event) COWA_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(p->bwd_main_start_event), st));
-  cowa_bwd_kernel<D, false><<<(unsigned)nblocks, 512, BwdSmem<D>::kBytes, st>>>(mq, mk, mv, mdo, mdk, mdv, mdq, a);
+  cowa_bwd_kernel<D, false><<<(unsigned)nblocks, 512, BwdSmem<D>::kBytes, st>>>(mq, mk, mv, mdo, mdk, mdv, a);
   COWA_CUDA_TRY(cudaGetLastError());
   if (p->bwd_main_stop_event) COWA_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(p->bwd_main_stop_event), st));
   {
@@ -966,12 +966,9 @@ int launch_bwd_varlen(const void* q, const void* k, const void* v, const void* o
   float* lse2 = dq_acc + (size_t)Hq * Tpad * D;
   float* delta = lse2 + (size_t)Hq * Tpad;
   if (cowa::any_stride_set(p)) return COWA_ERR_UNSUPPORTED;  // packed tensors are contiguous [H, total, D]
-  CUtensorMap mq, mk, mv, mdo, mdk, mdv, mdq;
+  CUtensorMap mq, mk, mv, mdo, mdk, mdv;
   int rc;
   const CowaStrides sq = packed_strides(Hq, total, D), sk = packed_strides(Hkv, total, D);
-  if ((rc = cowa::make_tensor_map(&mdq, dq_acc, p->deterministic ? cowa::MapType::S32 : cowa::MapType::F32, D, Tpad, Hq, 1,
-                                  packed_strides(Hq, Tpad, D), D, 32, false)))
-    return rc;
   if ((rc = cowa::make_tensor_map(&mq, q, cowa::MapType::BF16, D, total, Hq, 1, sq, 64, BQS))) return rc;
   if ((rc = cowa::make_tensor_map(&mdo, d_o, cowa::MapType::BF16, D, total, Hq, 1, sq, 64, BQS))) return rc;
   if ((rc = cowa::make_tensor_map(&mk, k, cowa::MapType::BF16, D, total, Hkv, 1, sk, 64, BKV))) return rc;
@@ -1009,7 +1006,7 @@ int launch_bwd_varlen(const void* q, const void* k, const void* v, const void* o
       static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse, lse2, delta, cu, B, total, Tpad);
   COWA_CUDA_TRY(cudaGetLastError());
   if (p->bwd_main_start_event) COWA_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(p->bwd_main_start_event), st));
-  cowa_bwd_kernel<D, true><<<(unsigned)nblocks, 512, BwdSmem<D>::kBytes, st>>>(mq, mk, mv, mdo, mdk, mdv, mdq, a);
+  cowa_bwd_kernel<D, true><<<(unsigned)nblocks, 512, BwdSmem<D>::kBytes, st>>>(mq, mk, mv, mdo, mdk, mdv, a);
   COWA_CUDA_TRY(cudaGetLastError());
   if (p->bwd_main_stop_event) COWA_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(p->bwd_main_stop_event), st));
   cowa_bwd_convert_dq_varlen_kernel<D><<<chunks, BQS * (D / 8), 0, st>>>(dq_acc, static_cast<__nv_bfloat16*>(dq), cu, B,
