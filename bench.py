@@ -252,6 +252,18 @@ def cpu_threads():
     return os.cpu_count() or 1
 
 
+def workload_config(args, world):
+    """The `config` object of the JSON line; both arms print the same one."""
+    import cowa_inputs
+    ct = cowa_inputs.CONFIGS[args.train_cfg]
+    cd = cowa_inputs.CONFIGS[DECODE_CFG]
+    return {"workload": args.train_cfg, "decode_workload": DECODE_CFG, "decode_batch": args.decode_batch or cd["B"],
+            "B": ct["B"], "T": ct["T"], "Hq": ct["Hq"], "Hkv": ct["Hkv"], "D": ct["D"], "sink": ct["sink"], "near": ct["local"],
+            "deterministic_dq": bool(args.deterministic), "windows": args.windows, "phases": ["fwd", "bwd", "decode"],
+            "l2": "inputs larger than L2 (2.6 GB training tensors, 0.57 GB visible KV cache)",
+            "parallelism": "independent replicas" if world > 1 else "single GPU"}
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -272,7 +284,7 @@ def run_reference(args):
         "impl": "reference", "metric": "cowa_train_tflops_visited_tiles_128k", "value": val, "unit": "TFLOP/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": TRAIN_CFG, "note": "float64 CPU oracle, legal-pair FLOPs of the sampled tiles"},
+        "config": workload_config(argparse.Namespace(**{**vars(args), "train_cfg": TRAIN_CFG}), args.gpus), "config_note": "float64 CPU oracle, legal-pair FLOPs of the sampled tiles",
         "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cpu_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -730,11 +742,7 @@ def run_cuda(args):
         "metric": "cowa_train_tflops_visited_tiles_" + args.train_cfg, "value": value, "unit": "TFLOP/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": args.train_cfg, "decode_workload": DECODE_CFG, "decode_batch": cd["B"], "B": B, "T": T, "Hq": Hq, "Hkv": Hkv,
-                   "D": D, "sink": ct["sink"], "near": ct["local"], "deterministic_dq": bool(args.deterministic), "windows": args.windows,
-                   "phases": ["fwd"] + (["bwd"] if have_bwd else []) + ["decode"],
-                   "l2": "inputs larger than L2 (2.6 GB training tensors, 0.57 GB visible KV cache)",
-                   "parallelism": "independent replicas" if world > 1 else "single GPU"},
+        "config": workload_config(args, world),
         "fwd_ms": fwd_ms, "fwd_ms_min": fwd_min, "fwd_tflops": fwd_flops / fwd_ms / 1e9,
         "fwd_tflops_legal_pairs": legal_pairs * 4 * D * G * B / fwd_ms / 1e9,
         "bwd_ms_min": bwd_min if have_bwd else None,
