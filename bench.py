@@ -836,6 +836,8 @@ def tp_replica_rows(cowa, cowa_inputs, dev, lengths, rank, world, warmup, iters)
     TP, Hq_r, D, sink, near = 8, 8, 128, 128, 896
     scale = cowa_inputs.softmax_scale(D)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    for _ in range(500):  # ~50 ms of memory traffic: the first microsecond-scale calls must not meet an idle GPU's clocks
+        flush.fill_(1)
     rows = []
     for T in lengths:
         q, k, v, d_o = cowa_inputs.make_train_inputs(11, 1, T, Hq_r, 1, D, device=dev)
